@@ -1,0 +1,491 @@
+#!/usr/bin/env python
+"""Benchmark of one suffix-pruned denoising step on B200.
+
+A step = ds_attn_pruned (once per resident layer cache) + ds_confidence +
+ds_unmask_select over one batch of seeded synthetic input.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+* ``value``: denoise steps/s with every input resident in HBM, timed with CUDA
+  events on the launching stream (max over ranks; ranks are independent replicas,
+  each with its own batch: weak scaling, no collective on the data path).
+* ``roofline``: the attention kernel's algorithmic bytes / its mean launch time
+  (CUDA events inside the timed region) against the measured HBM peak.
+* ``e2e``: the same step through the public API starting from pinned HOST
+  buffers: host->device copies of everything the step reads and device->host
+  copies of its results are inside the timed region.
+* ``cpu_baseline``: the CPU oracle, as it stands, timed on this machine's host
+  cores on a bounded sample of the same workload and scaled to a full step.
+* ``--impl reference`` times that oracle as the main line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "pruned-step attn+confidence: denoise steps/s"
+DEFAULT_CONFIG = "long32-w64"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (bytes; None until a capture of that kernel and workload exists)
+NCU_TRAFFIC: dict = {}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def attn_algorithmic_bytes(cfg, Lq):
+    e = 4 if cfg.dtype == "f32" else 2
+    kv_prefix = 2 * cfg.B * cfg.Hkv * cfg.P * cfg.D * e
+    kv_tail = 2 * cfg.B * cfg.Hkv * Lq * cfg.D * e
+    q = cfg.B * cfg.Hq * Lq * cfg.D * e
+    return kv_prefix + kv_tail + 2 * q          # + O, same size as Q
+
+
+def attn_flops(cfg, Lq):
+    return 4 * cfg.B * cfg.Hq * Lq * (cfg.P + Lq) * cfg.D
+
+
+def conf_algorithmic_bytes(cfg):
+    e = 4 if cfg.dtype == "f32" else 2
+    return cfg.rows * cfg.V * e + 8 * cfg.rows
+
+
+# --------------------------------------------------------------------------
+# clock sampling (read-only NVML)
+# --------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, torch_device_index: int, period_s: float = 0.004):
+        self.samples = []      # (t, sm_mhz, reasons bitmask)
+        self.period = period_s
+        self._stop = threading.Event()
+        self._thread = None
+        self.h = None
+        self.max_mhz = None
+        try:
+            import pynvml
+            import torch
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(torch_device_index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(torch_device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as exc:  # NVML missing: report that, do not fail the run
+            self.err = repr(exc)
+            self.h = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append((time.perf_counter(), mhz, rs))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self, windows):
+        if self.h is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable"}
+        sel = [s for s in self.samples if any(a <= s[0] <= b for a, b in windows)]
+        if not sel:
+            sel = self.samples
+        mhz = sorted(s[1] for s in sel)
+        mask = 0
+        for s in sel:
+            mask |= s[2]
+        reasons = [n for bit, n in self.REASONS.items() if mask & bit]
+        return {"sm_mhz": mhz[len(mhz) // 2] if mhz else None, "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(sel)}
+
+
+# --------------------------------------------------------------------------
+# the GPU step
+# --------------------------------------------------------------------------
+class Step:
+    """Device-resident inputs of one configuration and the three C-ABI calls of a step."""
+
+    def __init__(self, cfg, device, compact_tail=False):
+        import torch
+        import paper_2601_17917_b200 as ds
+        from paper_2601_17917_b200 import workloads as wl
+        self.torch, self.ds, self.cfg, self.device = torch, ds, cfg, device
+        idx = ds.retained_indices(cfg.gen, cfg.K, 0, cfg.w, cfg.keep_last)
+        self.Lq = len(idx)
+        self.layers = []
+        for layer in range(cfg.n_layers):
+            x = wl.attention_inputs(cfg, device=device, layer=layer)
+            if compact_tail:
+                sel = torch.tensor(idx, device=device)
+                for k in ("q_tail", "k_tail", "v_tail"):
+                    x[k] = x[k][:, :, sel].contiguous()
+            self.layers.append(x)
+        if compact_tail:
+            idx = list(range(self.Lq))
+        self.idx = torch.tensor(idx, dtype=torch.int32, device=device)
+        self.scale = 1.0 / math.sqrt(cfg.D)
+        self.logits = wl.logits(cfg, device=device)
+        x0, m0 = wl.block_state(cfg, "all")
+        self.x0, self.m0 = x0.to(device), m0.to(device)
+        self.x_block, self.masked = self.x0.clone(), self.m0.clone()
+        dt = cfg.torch_dtype()
+        B, K = cfg.B, cfg.K
+        self.out = torch.empty((B, cfg.Hq, self.Lq, cfg.D), dtype=dt, device=device)
+        self.conf = torch.empty(cfg.rows, dtype=torch.float32, device=device)
+        self.tok = torch.empty(cfg.rows, dtype=torch.int32, device=device)
+        self.sel = dict(sel_idx=torch.empty((B, K), dtype=torch.int32, device=device),
+                        sel_cnt=torch.zeros(B, dtype=torch.int32, device=device),
+                        block_done=torch.zeros(B, dtype=torch.uint8, device=device),
+                        eos_exit=torch.zeros(B, dtype=torch.uint8, device=device),
+                        active_seq=torch.empty(B, dtype=torch.int32, device=device),
+                        active_cnt=torch.zeros(1, dtype=torch.int32, device=device))
+        x = self.layers[0]
+        need = ds.ds_attn_pruned_workspace(x["q_tail"], x["k_tail"], x["v_tail"], x["k_pre"], x["v_pre"],
+                                           self.idx, self.scale, self.out)
+        self.attn_ws = torch.empty(max(need, 256), dtype=torch.uint8, device=device)
+        self.conf_ws = torch.empty(max(ds.ds_confidence_workspace(cfg.rows, cfg.V, dt), 256), dtype=torch.uint8,
+                                   device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def attn(self, layer=0):
+        x = self.layers[layer]
+        self.ds.ds_attn_pruned(x["q_tail"], x["k_tail"], x["v_tail"], x["k_pre"], x["v_pre"], self.idx, self.scale,
+                               out=self.out, workspace=self.attn_ws, status=self.status)
+
+    def confidence(self):
+        self.ds.ds_confidence(self.logits, conf=self.conf, tok=self.tok, workspace=self.conf_ws)
+
+    def select(self):
+        cfg = self.cfg
+        # every timed step starts from the same block state (two small device-to-device copies)
+        self.masked.copy_(self.m0)
+        self.x_block.copy_(self.x0)
+        self.ds.ds_unmask_select(self.conf.view(cfg.B, cfg.K), self.tok.view(cfg.B, cfg.K), self.masked, self.x_block,
+                                 cfg.tau0, cfg.alpha, eos_id=cfg.V - 2, eos_tau=cfg.tau0, out=self.sel)
+
+    def run(self, events=None):
+        """One whole step.  ``events``: optional [4] CUDA events recorded between the stages."""
+        if events:
+            events[0].record()
+        for layer in range(self.cfg.n_layers):
+            self.attn(layer)
+        if events:
+            events[1].record()
+        self.confidence()
+        if events:
+            events[2].record()
+        self.select()
+        if events:
+            events[3].record()
+
+
+def time_resident(step, steps, warmup, sampler, barrier):
+    torch = step.torch
+    for _ in range(warmup):
+        step.run()
+    torch.cuda.synchronize()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    barrier()
+    torch.cuda.synchronize()
+    launches0 = step.ds.ds_launch_count()
+    t0 = time.perf_counter()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(steps):
+        step.run(evs[i])
+    end.record()
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    barrier()
+    total_ms = start.elapsed_time(end)
+    launches = step.ds.ds_launch_count() - launches0
+    stage_ms = [sum(e[k].elapsed_time(e[k + 1]) for e in evs) / steps for k in range(3)]
+    windows = [(t0, t1)]
+    # the sampler needs a few samples under this load: if the timed region was short, run identical
+    # (untimed) steps for a moment longer
+    extra = 0
+    if sampler is not None and (t1 - t0) < 0.25:
+        t2 = time.perf_counter()
+        while time.perf_counter() - t2 < 0.3:
+            for _ in range(8):
+                step.run()
+            torch.cuda.synchronize()
+            extra += 8
+        windows.append((t2, time.perf_counter()))
+    return total_ms, stage_ms, launches, windows, extra
+
+
+def time_e2e(cfg, device, steps, warmup):
+    """Same step from pinned host buffers: H2D of everything the step reads, the three calls,
+    D2H of the results, all inside the timed region."""
+    import torch
+    dev_step = Step(cfg, device, compact_tail=True)
+    host_in, dev_in = [], []
+    for x in dev_step.layers:
+        for k in ("q_tail", "k_tail", "v_tail", "k_pre", "v_pre"):
+            dev_in.append(x[k])
+    dev_in += [dev_step.logits, dev_step.x_block, dev_step.masked, dev_step.idx]
+    for t in dev_in:
+        h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+        h.copy_(t)
+        host_in.append(h)
+    dev_out = [dev_step.out, dev_step.x_block, dev_step.masked, dev_step.sel["sel_idx"], dev_step.sel["sel_cnt"],
+               dev_step.sel["block_done"], dev_step.sel["eos_exit"], dev_step.sel["active_seq"],
+               dev_step.sel["active_cnt"]]
+    host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in dev_out]
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
+
+    def one():
+        for h, d in zip(host_in, dev_in):
+            d.copy_(h, non_blocking=True)
+        dev_step.run()
+        for h, d in zip(host_out, dev_out):
+            h.copy_(d, non_blocking=True)
+
+    for _ in range(max(1, min(warmup, 3))):
+        one()
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        one()
+    end.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(end) / steps, h2d, d2h
+
+
+# --------------------------------------------------------------------------
+# CPU oracle timing (baseline leg and --impl reference)
+# --------------------------------------------------------------------------
+class OracleSample:
+    """A bounded sample of the workload for the CPU oracle: ``n_slices`` (batch, head) attention
+    slices of one layer, ``n_rows`` logit rows, and the full selection.  ``time()`` runs the
+    oracle on it and returns the seconds a whole step would take at that rate (linear scaling over
+    slices, rows and layers)."""
+
+    def __init__(self, cfg, n_slices, n_rows):
+        import numpy as np
+        import oracle
+        from paper_2601_17917_b200 import workloads as wl
+        self.np, self.oracle, self.cfg = np, oracle, cfg
+        w = cfg.w if cfg.w >= 0 else cfg.gen
+        self.idx = np.asarray(oracle.retained_indices(cfg.gen, cfg.K, 0, w, cfg.keep_last))
+        n_slices = min(n_slices, cfg.B * cfg.Hq)
+        hs = min(cfg.Hq, n_slices)
+        bs = max(1, n_slices // hs)
+        G = cfg.Hq // cfg.Hkv
+        small = wl.shrink(cfg, B=bs, Hq=hs, Hkv=hs // G if hs % G == 0 else hs)
+        self.small = small
+        self.x = {k: v.float().numpy() for k, v in wl.attention_inputs(small, device="cpu").items()}
+        self.n_rows = min(n_rows, cfg.rows)
+        self.z = wl.logits(cfg, device="cpu", rows=self.n_rows).float().numpy()
+        self.conf = np.random.default_rng(0).random((cfg.B, cfg.K)).astype(np.float32)
+        self.tok = np.zeros((cfg.B, cfg.K), np.int32)
+        xb, mk = wl.block_state(cfg, "all")
+        self.xb, self.mk = xb.numpy(), mk.numpy()
+        self.scale = 1.0 / math.sqrt(cfg.D)
+        self.cores = oracle.num_threads()
+        self.sample = (f"{small.B * small.Hq} of {cfg.B * cfg.Hq} (batch, head) attention slices of one layer, "
+                       f"{self.n_rows} of {cfg.rows} logit rows, full selection; scaled linearly to one step"
+                       + (f" x {cfg.n_layers} layers" if cfg.n_layers > 1 else ""))
+
+    def time(self):
+        cfg, x, o = self.cfg, self.x, self.oracle
+        t0 = time.perf_counter()
+        o.attn(x["q_tail"], x["k_tail"], x["v_tail"], x["k_pre"], x["v_pre"], self.idx, self.scale)
+        t1 = time.perf_counter()
+        o.confidence(self.z)
+        t2 = time.perf_counter()
+        o.select(self.conf, self.tok, self.mk, self.xb, cfg.tau0, cfg.alpha)
+        t3 = time.perf_counter()
+        full = ((t1 - t0) * (cfg.B * cfg.Hq) / (self.small.B * self.small.Hq) * cfg.n_layers
+                + (t2 - t1) * cfg.rows / self.n_rows + (t3 - t2))
+        return full, t3 - t0
+
+
+def run_reference(args, cfg):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    smp = OracleSample(cfg, 32, 256)
+    for _ in range(min(args.warmup, 1)):
+        smp.time()
+    times = []
+    t_all0 = time.perf_counter()
+    for _ in range(max(args.steps, 1)):
+        times.append(smp.time()[0])
+        if time.perf_counter() - t_all0 > 150:       # bounded: a few minutes at most
+            break
+    sec = sum(times) / len(times)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": 1.0 / sec, "unit": "steps/s", "n_gpus": args.gpus,
+        "steps": len(times), "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D, "P": cfg.P,
+                   "gen": cfg.gen, "K": cfg.K, "Lq": int(len(smp.idx)), "V": cfg.V, "n_layers": cfg.n_layers},
+        "cpu_baseline": {"value": 1.0 / sec, "unit": "steps/s", "cores": smp.cores, "kind": "oracle",
+                         "sample": smp.sample},
+        "e2e": {"value": 1.0 / sec, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", default=DEFAULT_CONFIG)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2601_17917_b200 import workloads as wl
+    cfg = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2601_17917_b200 as ds
+    ds.lib()                     # fail loudly if the CUDA library is not built: there is no fallback
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback exists)")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    warmup = max(args.warmup, 3)
+    # replicas: every rank draws its own batch (its rank offsets the seed); no data-path collective
+    rcfg = wl.shrink(cfg, seed=cfg.seed + 100000 * rank)
+    step = Step(rcfg, device)
+    sampler = ClockSampler(local)
+    sampler.start()
+    total_ms, stage_ms, launches, windows, extra = time_resident(step, args.steps, warmup, sampler, barrier)
+    sampler.stop()
+    clocks = sampler.summary(windows)
+    if extra:
+        clocks["note"] = f"timed region + {extra} further identical steps"
+    status = ds.ds_read_status(step.status)
+    if world > 1:
+        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * 1e3 / ms_per_step
+
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(3, min(args.steps, 20))
+        del step.layers[1:]
+        torch.cuda.empty_cache()
+        e_ms, h2d, d2h = time_e2e(rcfg, device, e2e_steps, 3)
+        if world > 1:
+            t = torch.tensor([e_ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": world * 1e3 / e_ms, "unit": "steps/s", "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": e_ms, "steps": e2e_steps,
+               "layout": "tail rows shipped compact (T = Lq): only what the step reads crosses the link"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    Lq = step.Lq
+    a_bytes = attn_algorithmic_bytes(cfg, Lq)
+    a_ms = stage_ms[0] / cfg.n_layers
+    a_gbs = a_bytes / (a_ms * 1e-3) / 1e9
+    c_bytes = conf_algorithmic_bytes(cfg)
+    c_gbs = c_bytes / (stage_ms[1] * 1e-3) / 1e9
+    fl = attn_flops(cfg, Lq)
+    traffic = NCU_TRAFFIC.get(cfg.name, {})
+    line = {
+        "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D, "P": cfg.P,
+                   "gen": cfg.gen, "K": cfg.K, "window_tokens": cfg.w, "Lq": Lq, "Lkv": cfg.P + Lq, "V": cfg.V,
+                   "n_layers": cfg.n_layers, "tau0": cfg.tau0, "alpha": cfg.alpha, "parallelism": f"replicas x{world}",
+                   "l2": "inputs larger than L2 (KV cache and logits of one step exceed 126 MB)"
+                   if a_bytes * cfg.n_layers + c_bytes > 2 * 126e6 else "working set near L2 size"},
+        "tokens_per_s": {"query_tokens": value * cfg.B * Lq,
+                         "committed_tokens": value * float(step.sel["sel_cnt"].sum().item())},
+        "stage_ms": {"attn_per_layer": a_ms, "confidence": stage_ms[1], "select": stage_ms[2]},
+        "roofline": {"kernel": "ds_attn_pruned", "bound": "hbm", "achieved": a_gbs, "peak": pk["hbm_gbs"],
+                     "unit": "GB/s", "frac": a_gbs / pk["hbm_gbs"], "traffic": traffic.get("attn_bytes_per_launch"),
+                     "peak_source": pk["_source"], "algorithmic_bytes": a_bytes,
+                     "tflops": fl / (a_ms * 1e-3) / 1e12,
+                     "tensor_frac_of_sustained": fl / (a_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"]},
+        "roofline_confidence": {"kernel": "ds_confidence", "bound": "hbm", "achieved": c_gbs, "peak": pk["hbm_gbs"],
+                                "unit": "GB/s", "frac": c_gbs / pk["hbm_gbs"],
+                                "traffic": traffic.get("confidence_bytes_per_launch"), "peak_source": pk["_source"],
+                                "algorithmic_bytes": c_bytes},
+        "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
+    }
+    if e2e:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        smp = OracleSample(cfg, 64, 512)
+        full_s, spent = smp.time()
+        line["cpu_baseline"] = {"value": 1.0 / full_s, "unit": "steps/s", "cores": smp.cores, "kind": "oracle",
+                                "sample": smp.sample, "sample_seconds": spent}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

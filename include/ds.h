@@ -1,0 +1,208 @@
+/*
+ * ds.h -- C ABI of the B200 (sm_100a) suffix-pruned denoising step.
+ *
+ * One step of block-diffusion decoding with attenuation-guided suffix pruning
+ * and dynamic confidence-aware unmasking has three device stages:
+ *
+ *   ds_attn_pruned    bidirectional attention of {current block U retained
+ *                     suffix rows} over {cached prefix KV ; the same retained
+ *                     rows}  (Method, Eq. 7 and Eq. 8, and the query/key
+ *                     construction of "Dynamic Confidence Aware Parallel
+ *                     Decoding")
+ *   ds_confidence     c = max softmax(z), x^ = argmax softmax(z) per logit row
+ *                     (Preliminary, Eq. 4)
+ *   ds_unmask_select  adaptive threshold (Eq. 10), selection rule (Eq. 9),
+ *                     state update (Eq. 5), block-finished test and the
+ *                     early-exit flag ("Early Exit For Block Diffusion")
+ *
+ * Conventions
+ *   - Every function returns a ds_status.  Nothing throws, traps or aborts.
+ *   - Unless a parameter is marked HOST, pointers are DEVICE pointers on the
+ *     current CUDA device.  The caller owns every buffer; the library never
+ *     allocates or frees device memory and never synchronises a stream (except
+ *     ds_read_status, which says so).  Work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - Shapes outside a kernel's envelope return DS_ERR_UNSUPPORTED; there is
+ *     no CPU fallback.
+ *   - Conditions only the device can see (a retained-row index out of range, a
+ *     bounded on-chip wait that ran out) are OR-ed into the optional device
+ *     word `status` as DS_DEV_* bits; the kernel still terminates normally.
+ *   - Calls on distinct streams may run concurrently provided they do not
+ *     share a workspace.
+ */
+#ifndef DS_H_
+#define DS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DS_API __attribute__((visibility("default")))
+#else
+#define DS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DS_OK = 0,
+  DS_ERR_INVALID_ARG = 1, /* null pointer, negative size, inconsistent shape, misaligned pointer/stride */
+  DS_ERR_UNSUPPORTED = 2, /* well-formed request outside the kernels' envelope */
+  DS_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or smaller than the *_workspace() query */
+  DS_ERR_CUDA = 4         /* a CUDA runtime/driver call failed (launch, tensor-map encode, ...) */
+} ds_status;
+
+/* bits OR-ed into the optional device status word */
+#define DS_DEV_INDEX 1u   /* an entry of idx was outside [0, T); it was clamped */
+#define DS_DEV_TIMEOUT 2u /* a bounded mbarrier wait expired; outputs of that CTA are invalid */
+
+typedef enum { DS_F32 = 0, DS_BF16 = 1 } ds_dtype;
+
+/* ------------------------------------------------------------------------
+ * ds_attn_pruned  (Eq. 7, Eq. 8; "Dynamic Confidence Aware Parallel Decoding")
+ *
+ * The sequence at a denoising step is [prefix ; current block ; suffix]
+ * (Method, region split).  The "tail" is block + suffix, T rows.  The retained
+ * set of Eq. 7 arrives as `idx`: Lq tail-relative row numbers, strictly
+ * ascending (block rows first, then the window, then the trailing position).
+ * For every batch b and query head h, with KV head g = h / (Hq / Hkv):
+ *
+ *     Q~ = q_tail[b, h, idx[:], :]                          (Lq x D)
+ *     K~ = [ k_prefix[b, g, 0:P, :] ; k_tail[b, g, idx[:], :] ]   ((P + Lq) x D)
+ *     V~ likewise
+ *     out[b, h, i, :] = sum_j softmax_j(scale * <Q~_i, K~_j>) V~_j
+ *
+ * There is no mask: the model is bidirectional.  Rotary position encoding is
+ * applied by the caller (pruned rows keep their original position ids).
+ * Accumulation is fp32; `out` has the input element type.  `lse`, when not
+ * NULL, receives log(sum_j exp(scale * <Q~_i, K~_j>)) (natural log, fp32).
+ *
+ * Layout: element strides (not bytes) for the batch, head and row dimensions;
+ * the D dimension is contiguous.  Every base pointer must be 16-byte aligned
+ * and every stride a multiple of 16 bytes (8 bf16 / 4 fp32 elements).  P may be 0 (the
+ * prefix pointers are then ignored).  idx is either one list shared by all
+ * batches (idx_batch_stride = 0) or one per batch.
+ *
+ * Envelope: D in {64, 128} for the tensor-core bf16 path; the fp32 path takes
+ * any D that is a multiple of 32 up to 256.  Hq % Hkv == 0.  1 <= Lq <= T.
+ *
+ * Workspace: ds_attn_pruned_workspace(p) bytes, 256-byte aligned, used for
+ * split-KV partial results; contents need not be preserved between calls.
+ * Errors: DS_ERR_INVALID_ARG / DS_ERR_UNSUPPORTED / DS_ERR_WORKSPACE before
+ * anything is launched; DS_ERR_CUDA if a launch fails.
+ * ------------------------------------------------------------------------ */
+typedef struct {
+  int32_t B, Hq, Hkv, D;
+  int32_t P;  /* cached prefix length (prompt + decoded blocks), >= 0 */
+  int32_t T;  /* rows in the tail buffers */
+  int32_t Lq; /* retained rows: K + R */
+  int32_t dtype; /* ds_dtype of q/k/v/out */
+  const void *q_tail;                /* [B][Hq ][T][D] */
+  const void *k_tail, *v_tail;       /* [B][Hkv][T][D] */
+  const void *k_prefix, *v_prefix;   /* [B][Hkv][P][D] */
+  int64_t q_stride[3];               /* batch, head, row (elements) */
+  int64_t kv_tail_stride[3];
+  int64_t kv_prefix_stride[3];
+  int64_t out_stride[3];
+  const int32_t *idx;                /* [Lq] or [B][Lq] */
+  int64_t idx_batch_stride;          /* 0 or >= Lq */
+  float scale;                       /* softmax scale, 1/sqrt(D) for the standard definition */
+  void *out;                         /* [B][Hq][Lq][D] */
+  float *lse;                        /* optional [B][Hq][Lq], dense */
+  void *workspace;
+  size_t workspace_bytes;
+  uint32_t *status;                  /* optional device word, DS_DEV_* bits are OR-ed in */
+} ds_attn_params;
+
+/* HOST, pure: bytes of workspace ds_attn_pruned needs for *p (0 when none). */
+DS_API size_t ds_attn_pruned_workspace(const ds_attn_params *p);
+/* `p` is a HOST pointer; the pointers inside it are device pointers. */
+DS_API int ds_attn_pruned(const ds_attn_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
+ * ds_confidence  (Eq. 4)
+ *
+ * For every selected row r of logits[rows][V] (row stride ld >= V elements):
+ *     m       = max_j z_rj
+ *     tok[r]  = lowest j with z_rj == m
+ *     conf[r] = 1 / sum_j exp(z_rj - m)          (= max_j softmax(z_r)_j)
+ * computed in fp32 from one read of the row.  `row_list` (n_listed ascending
+ * row numbers) restricts the pass to those rows, e.g. the still-masked
+ * positions; NULL means all rows.  conf/tok are indexed by row number; rows
+ * not listed are left untouched.
+ *
+ * Workspace: ds_confidence_workspace(rows, V, dtype) bytes, 256-byte aligned;
+ * used when a row is split over several CTAs (few rows, large V).  The
+ * library clears the part it needs on `stream` before the kernel runs.
+ * ------------------------------------------------------------------------ */
+DS_API size_t ds_confidence_workspace(int64_t rows, int64_t V, int32_t dtype);
+DS_API int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_t V, int64_t ld,
+                  const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
+                  void *workspace, size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------
+ * ds_unmask_select  (Eq. 9, Eq. 10, Eq. 5, block termination, early exit)
+ *
+ * Per processed sequence b, with n = number of masked positions of its block
+ * BEFORE this step:
+ *     r_mask = (n + ratio_extra) / (K + ratio_extra)
+ *     tau    = tau0 * (1 - alpha * (1 - r_mask))           (fp32, one rounding per op)
+ *     accept = { i : masked[b][i] and conf[b][i] >= tau }
+ *     if accept is empty and n > 0: accept = { lowest i among masked with maximal conf }
+ *     for i in accept: x_block[b][i] = tok[b][i]; masked[b][i] = 0
+ *     sel_idx[b][0:sel_cnt[b]] = accept ascending, remaining entries -1
+ *     block_done[b] = 1 when no masked position is left, else 0
+ *     eos_exit[b]  |= 1 when an accepted token equals eos_id with conf >= eos_tau
+ *     active_seq    = ascending list of processed sequences with block_done == 0,
+ *                     *active_cnt its length
+ * ratio_extra = 0 counts the block only; ratio_extra = R also counts the
+ * retained suffix rows of the query (all still masked).  alpha = 0 gives the
+ * fixed-threshold rule.  eos_id < 0 disables the early-exit flag.
+ * seq_list (n_seq ascending sequence numbers, e.g. the previous step's
+ * active_seq) restricts processing; NULL = all B.  With seq_list, n_seq may be
+ * given as a device scalar instead (n_seq_dev != NULL overrides n_seq as the
+ * count, n_seq then being only the upper bound used to size the launch).
+ * Unprocessed sequences' outputs are left untouched.
+ * ------------------------------------------------------------------------ */
+typedef struct {
+  int32_t B, K;                 /* 1 <= K <= 4096 */
+  const float *conf;            /* [B][K] */
+  const int32_t *tok;           /* [B][K] */
+  uint8_t *masked;              /* [B][K] in/out, non-zero = still MASK */
+  int32_t *x_block;             /* [B][K] in/out */
+  float tau0, alpha;
+  int32_t ratio_extra;          /* >= 0 */
+  int32_t eos_id;
+  float eos_tau;
+  const int32_t *seq_list;      /* optional [n_seq] */
+  int32_t n_seq;
+  const int32_t *n_seq_dev;     /* optional device scalar */
+  int32_t *sel_idx;             /* [B][K] */
+  int32_t *sel_cnt;             /* [B] */
+  uint8_t *block_done;          /* [B] */
+  uint8_t *eos_exit;            /* [B] in/out */
+  int32_t *active_seq;          /* [B] */
+  int32_t *active_cnt;          /* [1] */
+} ds_select_params;
+
+/* `p` is a HOST pointer; the pointers inside it are device pointers. */
+DS_API int ds_unmask_select(const ds_select_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Utilities
+ * ------------------------------------------------------------------------ */
+/* Copies the device status word to *host_out (HOST) after synchronising `stream`. */
+DS_API int ds_read_status(const uint32_t *device_status, void *stream, uint32_t *host_out);
+/* HOST: static string for a ds_status value. */
+DS_API const char *ds_strerror(int code);
+/* HOST: library version, major * 1000 + minor. */
+DS_API int ds_version(void);
+/* HOST: number of kernels this library has launched in this process (all entry points). */
+DS_API int64_t ds_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DS_H_ */

@@ -1,0 +1,279 @@
+"""B200-native suffix-pruned denoising step for block-diffusion LLM decoding.
+
+Thin Python binding over the C-ABI library ``libds_b200.so`` (declared in
+``include/ds.h``).  The functions here have the same names as the C entry
+points and only marshal arguments: torch tensors supply device memory and the
+current stream, every step of the path runs in the library's CUDA kernels.
+There is no CPU or PyTorch fallback: if the library is not built, importing
+succeeds but the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+from . import workloads  # noqa: F401  (seeded synthetic inputs)
+
+__all__ = [
+    "lib", "retained_indices", "ds_attn_pruned", "ds_attn_pruned_workspace", "ds_confidence",
+    "ds_confidence_workspace", "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
+    "ds_launch_count", "DsError", "DS_F32", "DS_BF16", "DS_DEV_INDEX", "DS_DEV_TIMEOUT",
+]
+
+DS_F32, DS_BF16 = 0, 1
+DS_OK, DS_ERR_INVALID_ARG, DS_ERR_UNSUPPORTED, DS_ERR_WORKSPACE, DS_ERR_CUDA = range(5)
+DS_DEV_INDEX, DS_DEV_TIMEOUT = 1, 2
+
+_LIB_PATH = Path(__file__).resolve().parent / "libds_b200.so"
+_lib = None
+
+
+class DsError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {ds_strerror(code)} (status {code})")
+
+
+class _AttnParams(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32),
+        ("P", ctypes.c_int32), ("T", ctypes.c_int32), ("Lq", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("q_tail", ctypes.c_void_p), ("k_tail", ctypes.c_void_p), ("v_tail", ctypes.c_void_p),
+        ("k_prefix", ctypes.c_void_p), ("v_prefix", ctypes.c_void_p),
+        ("q_stride", ctypes.c_int64 * 3), ("kv_tail_stride", ctypes.c_int64 * 3),
+        ("kv_prefix_stride", ctypes.c_int64 * 3), ("out_stride", ctypes.c_int64 * 3),
+        ("idx", ctypes.c_void_p), ("idx_batch_stride", ctypes.c_int64), ("scale", ctypes.c_float),
+        ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t), ("status", ctypes.c_void_p),
+    ]
+
+
+class _SelectParams(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("K", ctypes.c_int32), ("conf", ctypes.c_void_p), ("tok", ctypes.c_void_p),
+        ("masked", ctypes.c_void_p), ("x_block", ctypes.c_void_p), ("tau0", ctypes.c_float),
+        ("alpha", ctypes.c_float), ("ratio_extra", ctypes.c_int32), ("eos_id", ctypes.c_int32),
+        ("eos_tau", ctypes.c_float), ("seq_list", ctypes.c_void_p), ("n_seq", ctypes.c_int32),
+        ("n_seq_dev", ctypes.c_void_p), ("sel_idx", ctypes.c_void_p), ("sel_cnt", ctypes.c_void_p),
+        ("block_done", ctypes.c_void_p), ("eos_exit", ctypes.c_void_p), ("active_seq", ctypes.c_void_p),
+        ("active_cnt", ctypes.c_void_p),
+    ]
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2601_17917_b200.build` "
+                               "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        L.ds_attn_pruned_workspace.restype = ctypes.c_size_t
+        L.ds_attn_pruned_workspace.argtypes = [ctypes.POINTER(_AttnParams)]
+        L.ds_attn_pruned.restype = ctypes.c_int
+        L.ds_attn_pruned.argtypes = [ctypes.POINTER(_AttnParams), ctypes.c_void_p]
+        L.ds_confidence_workspace.restype = ctypes.c_size_t
+        L.ds_confidence_workspace.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int32]
+        L.ds_confidence.restype = ctypes.c_int
+        L.ds_confidence.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                    ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                                    ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.ds_unmask_select.restype = ctypes.c_int
+        L.ds_unmask_select.argtypes = [ctypes.POINTER(_SelectParams), ctypes.c_void_p]
+        L.ds_read_status.restype = ctypes.c_int
+        L.ds_read_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
+        L.ds_strerror.restype = ctypes.c_char_p
+        L.ds_strerror.argtypes = [ctypes.c_int]
+        L.ds_version.restype = ctypes.c_int
+        L.ds_launch_count.restype = ctypes.c_int64
+        _lib = L
+    return _lib
+
+
+def ds_strerror(code: int) -> str:
+    return lib().ds_strerror(int(code)).decode()
+
+
+def ds_version() -> int:
+    return int(lib().ds_version())
+
+
+def ds_launch_count() -> int:
+    return int(lib().ds_launch_count())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return DS_F32
+    if t.dtype == torch.bfloat16:
+        return DS_BF16
+    raise TypeError(f"unsupported element type {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check_dev(*ts):
+    for t in ts:
+        if t is not None and not t.is_cuda:
+            raise ValueError("all tensors must live on a CUDA device")
+
+
+def retained_indices(gen_len: int, K: int, c: int, w_tokens: int, keep_last: bool = True) -> list[int]:
+    """Host step of the path: the retained set of Eq. 7 as tail-relative rows.
+
+    The tail starts at the current block c and has T = gen_len - c*K rows.
+    Kept: the K block rows, the next ``w_tokens`` rows (sliding window nearest
+    the block; -1 keeps the whole suffix), and the trailing position T-1.  The
+    list is strictly ascending, as ``ds_attn_pruned`` requires.
+    """
+    T = gen_len - c * K
+    if K <= 0 or T < K or w_tokens < -1:
+        raise ValueError("bad block / window")
+    end = T if w_tokens < 0 else min(K + w_tokens, T)
+    idx = list(range(end))
+    if keep_last and end < T:
+        idx.append(T - 1)
+    return idx
+
+
+def _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status):
+    B, Hq, T, D = q_tail.shape
+    Hkv = k_tail.shape[1]
+    P = 0 if k_prefix is None else k_prefix.shape[2]
+    for t in (q_tail, k_tail, v_tail, out) + ((k_prefix, v_prefix) if P else ()):
+        if t.stride(-1) != 1:
+            raise ValueError("the head dimension must be contiguous")
+    if k_tail.stride() != v_tail.stride() or (P and k_prefix.stride() != v_prefix.stride()):
+        raise ValueError("K and V must share strides")
+    if idx.dtype != torch.int32:
+        raise TypeError("idx must be int32")
+    Lq = idx.shape[-1]
+    p = _AttnParams()
+    p.B, p.Hq, p.Hkv, p.D, p.P, p.T, p.Lq = B, Hq, Hkv, D, P, T, Lq
+    p.dtype = _dtype_code(q_tail)
+    p.q_tail, p.k_tail, p.v_tail = q_tail.data_ptr(), k_tail.data_ptr(), v_tail.data_ptr()
+    p.k_prefix = k_prefix.data_ptr() if P else None
+    p.v_prefix = v_prefix.data_ptr() if P else None
+    p.q_stride[:] = q_tail.stride()[:3]
+    p.kv_tail_stride[:] = k_tail.stride()[:3]
+    if P:
+        p.kv_prefix_stride[:] = k_prefix.stride()[:3]
+    p.out_stride[:] = out.stride()[:3]
+    p.idx = idx.data_ptr()
+    p.idx_batch_stride = 0 if idx.dim() == 1 else idx.stride(0)
+    p.scale = float(scale)
+    p.out = out.data_ptr()
+    p.lse = lse.data_ptr() if lse is not None else None
+    p.workspace = workspace.data_ptr() if workspace is not None else None
+    p.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    p.status = status.data_ptr() if status is not None else None
+    return p
+
+
+def ds_attn_pruned_workspace(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out) -> int:
+    p = _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, None, None, None)
+    return int(lib().ds_attn_pruned_workspace(ctypes.byref(p)))
+
+
+def ds_attn_pruned(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out=None, lse=None,
+                   workspace=None, status=None, stream=None):
+    """Pruned attention (Eq. 7-8).  q_tail [B,Hq,T,D]; k_tail, v_tail [B,Hkv,T,D];
+    k_prefix, v_prefix [B,Hkv,P,D] or None; idx int32 [Lq] or [B,Lq] on the device.
+    Returns ``out`` [B,Hq,Lq,D].  Allocates ``out``/``workspace`` with torch when not given."""
+    _check_dev(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, out, lse, workspace, status)
+    B, Hq, T, D = q_tail.shape
+    if out is None:
+        out = torch.empty((B, Hq, idx.shape[-1], D), dtype=q_tail.dtype, device=q_tail.device)
+    p = _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status)
+    if workspace is None:
+        need = int(lib().ds_attn_pruned_workspace(ctypes.byref(p)))
+        if need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=q_tail.device)
+            p.workspace, p.workspace_bytes = workspace.data_ptr(), need
+    rc = lib().ds_attn_pruned(ctypes.byref(p), _stream(stream))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_attn_pruned")
+    return out
+
+
+def ds_confidence_workspace(rows: int, V: int, dtype) -> int:
+    code = dtype if isinstance(dtype, int) else (DS_BF16 if dtype == torch.bfloat16 else DS_F32)
+    return int(lib().ds_confidence_workspace(int(rows), int(V), code))
+
+
+def ds_confidence(logits, row_list=None, conf=None, tok=None, workspace=None, stream=None):
+    """Eq. 4 over ``logits`` [rows, V] (last dimension contiguous).  Returns (conf f32 [rows], tok i32 [rows])."""
+    _check_dev(logits, row_list, conf, tok, workspace)
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits must be [rows, V] with contiguous rows")
+    rows, V = logits.shape
+    if conf is None:
+        conf = torch.empty(rows, dtype=torch.float32, device=logits.device)
+    if tok is None:
+        tok = torch.empty(rows, dtype=torch.int32, device=logits.device)
+    if workspace is None:
+        need = ds_confidence_workspace(rows, V, logits.dtype)
+        workspace = torch.empty(max(need, 1), dtype=torch.uint8, device=logits.device)
+    if row_list is not None and row_list.dtype != torch.int32:
+        raise TypeError("row_list must be int32")
+    rc = lib().ds_confidence(_ptr(logits), _dtype_code(logits), rows, V, logits.stride(0), _ptr(row_list),
+                             0 if row_list is None else row_list.numel(), _ptr(conf), _ptr(tok),
+                             _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_confidence")
+    return conf, tok
+
+
+def ds_unmask_select(conf, tok, masked, x_block, tau0, alpha, ratio_extra=0, eos_id=-1, eos_tau=0.9,
+                     seq_list=None, n_seq=None, n_seq_dev=None, out=None, stream=None):
+    """Eq. 9-10 selection step.  conf f32 [B,K], tok i32 [B,K]; masked u8 [B,K] and
+    x_block i32 [B,K] are updated in place.  Returns a dict of device tensors:
+    sel_idx, sel_cnt, block_done, eos_exit, active_seq, active_cnt (pass ``out`` to reuse them)."""
+    _check_dev(conf, tok, masked, x_block, seq_list, n_seq_dev)
+    B, K = conf.shape
+    dev = conf.device
+    for t, dt in ((conf, torch.float32), (tok, torch.int32), (masked, torch.uint8), (x_block, torch.int32)):
+        if t.dtype != dt or not t.is_contiguous() or tuple(t.shape) != (B, K):
+            raise ValueError("conf/tok/masked/x_block must be contiguous [B,K] of f32/i32/u8/i32")
+    if out is None:
+        out = dict(sel_idx=torch.empty((B, K), dtype=torch.int32, device=dev),
+                   sel_cnt=torch.zeros(B, dtype=torch.int32, device=dev),
+                   block_done=torch.zeros(B, dtype=torch.uint8, device=dev),
+                   eos_exit=torch.zeros(B, dtype=torch.uint8, device=dev),
+                   active_seq=torch.empty(max(B, 1), dtype=torch.int32, device=dev),
+                   active_cnt=torch.zeros(1, dtype=torch.int32, device=dev))
+    p = _SelectParams()
+    p.B, p.K = B, K
+    p.conf, p.tok, p.masked, p.x_block = conf.data_ptr(), tok.data_ptr(), masked.data_ptr(), x_block.data_ptr()
+    p.tau0, p.alpha, p.ratio_extra, p.eos_id, p.eos_tau = tau0, alpha, ratio_extra, eos_id, eos_tau
+    if seq_list is not None:
+        if seq_list.dtype != torch.int32:
+            raise TypeError("seq_list must be int32")
+        # an empty tensor has a null data pointer, which the C ABI reads as "no list": keep it non-null
+        p.seq_list = seq_list.data_ptr() if seq_list.numel() else out["active_cnt"].data_ptr()
+        p.n_seq = seq_list.numel() if n_seq is None else min(int(n_seq), seq_list.numel())
+        p.n_seq_dev = n_seq_dev.data_ptr() if n_seq_dev is not None else None
+    p.sel_idx, p.sel_cnt = out["sel_idx"].data_ptr(), out["sel_cnt"].data_ptr()
+    p.block_done, p.eos_exit = out["block_done"].data_ptr(), out["eos_exit"].data_ptr()
+    p.active_seq, p.active_cnt = out["active_seq"].data_ptr(), out["active_cnt"].data_ptr()
+    rc = lib().ds_unmask_select(ctypes.byref(p), _stream(stream))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_unmask_select")
+    return out
+
+
+def ds_read_status(status: torch.Tensor, stream=None) -> int:
+    host = ctypes.c_uint32(0)
+    rc = lib().ds_read_status(_ptr(status), _stream(stream), ctypes.byref(host))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_read_status")
+    return int(host.value)

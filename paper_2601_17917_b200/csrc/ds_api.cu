@@ -1,0 +1,153 @@
+// C ABI of the denoising-step library: argument validation and dispatch.
+// Every step of the path runs in the CUDA kernels of the sibling files.
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+
+#include "ds_common.cuh"
+
+namespace ds {
+
+static std::atomic<long long> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int sm_count() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+namespace {
+
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int validate_attn(const ds_attn_params *p) {
+  if (!p) return DS_ERR_INVALID_ARG;
+  if (p->dtype != DS_F32 && p->dtype != DS_BF16) return DS_ERR_INVALID_ARG;
+  if (p->B < 0 || p->Hq <= 0 || p->Hkv <= 0 || p->D <= 0 || p->P < 0 || p->T <= 0) return DS_ERR_INVALID_ARG;
+  if (p->Hq % p->Hkv != 0) return DS_ERR_INVALID_ARG;
+  if (p->Lq < 1 || p->Lq > p->T) return DS_ERR_INVALID_ARG;
+  if (!p->q_tail || !p->k_tail || !p->v_tail || !p->idx || !p->out) return DS_ERR_INVALID_ARG;
+  if (p->P > 0 && (!p->k_prefix || !p->v_prefix)) return DS_ERR_INVALID_ARG;
+  if (p->idx_batch_stride != 0 && p->idx_batch_stride < p->Lq) return DS_ERR_INVALID_ARG;
+  if (!(p->scale == p->scale)) return DS_ERR_INVALID_ARG;
+  const int64_t unit = (p->dtype == DS_BF16) ? 8 : 4;  // 16 bytes
+  const void *ptrs[] = {p->q_tail, p->k_tail, p->v_tail, p->out, p->P > 0 ? p->k_prefix : nullptr,
+                        p->P > 0 ? p->v_prefix : nullptr};
+  for (const void *q : ptrs)
+    if (q && !aligned(q, 16)) return DS_ERR_INVALID_ARG;
+  if (!aligned(p->idx, 4) || (p->lse && !aligned(p->lse, 4)) || (p->status && !aligned(p->status, 4)))
+    return DS_ERR_INVALID_ARG;
+  const int64_t *strides[] = {p->q_stride, p->kv_tail_stride, p->out_stride, p->kv_prefix_stride};
+  for (int k = 0; k < 4; ++k) {
+    if (k == 3 && p->P == 0) continue;
+    for (int d = 0; d < 3; ++d) {
+      const int64_t s = strides[k][d];
+      if (s < 0 || s % unit != 0) return DS_ERR_INVALID_ARG;
+    }
+    if (strides[k][2] < p->D) return DS_ERR_INVALID_ARG;  // rows must not overlap
+  }
+  if (p->D % 32 != 0 || p->D > 256) return DS_ERR_UNSUPPORTED;
+  if (p->B > 65535 || p->Hq > 65535) return DS_ERR_UNSUPPORTED;
+  return DS_OK;
+}
+
+enum class AttnPath { kAuto, kSimt, kTc };
+AttnPath forced_path() {
+  const char *e = std::getenv("DS_ATTN_PATH");
+  if (!e) return AttnPath::kAuto;
+  if (!std::strcmp(e, "simt")) return AttnPath::kSimt;
+  if (!std::strcmp(e, "tc")) return AttnPath::kTc;
+  return AttnPath::kAuto;
+}
+
+}  // namespace
+}  // namespace ds
+
+extern "C" {
+
+size_t ds_attn_pruned_workspace(const ds_attn_params *p) {
+  if (ds::validate_attn(p) != DS_OK) return 0;
+  if (ds::forced_path() != ds::AttnPath::kSimt && ds::attn_tc_supported(*p)) return ds::attn_tc_workspace_bytes(*p);
+  return 0;
+}
+
+int ds_attn_pruned(const ds_attn_params *p, void *stream) {
+  const int rc = ds::validate_attn(p);
+  if (rc != DS_OK) return rc;
+  if (p->B == 0) return DS_OK;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const ds::AttnPath path = ds::forced_path();
+  const bool tc_ok = ds::attn_tc_supported(*p);
+  if (path == ds::AttnPath::kTc && !tc_ok) return DS_ERR_UNSUPPORTED;
+  if (tc_ok && path != ds::AttnPath::kSimt) {
+    const size_t need = ds::attn_tc_workspace_bytes(*p);
+    if (need > 0 && (!p->workspace || !ds::aligned(p->workspace, 256) || p->workspace_bytes < need))
+      return DS_ERR_WORKSPACE;
+    return ds::launch_attn_tc(*p, st);
+  }
+  return ds::launch_attn_simt(*p, st);
+}
+
+size_t ds_confidence_workspace(int64_t rows, int64_t V, int32_t dtype) {
+  if (dtype != DS_F32 && dtype != DS_BF16) return 0;
+  return ds::confidence_workspace_bytes(rows, V, dtype);
+}
+
+int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_t V, int64_t ld,
+                  const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok, void *workspace,
+                  size_t workspace_bytes, void *stream) {
+  if (dtype != DS_F32 && dtype != DS_BF16) return DS_ERR_INVALID_ARG;
+  if (rows < 0 || V <= 0 || ld < V || V > 0x7fffffffLL) return DS_ERR_INVALID_ARG;
+  if (rows == 0) return DS_OK;
+  if (!logits || !conf || !tok) return DS_ERR_INVALID_ARG;
+  const size_t esz = dtype == DS_BF16 ? 2 : 4;
+  if (!ds::aligned(logits, esz) || !ds::aligned(conf, 4) || !ds::aligned(tok, 4)) return DS_ERR_INVALID_ARG;
+  if (row_list && (n_listed < 0 || n_listed > rows)) return DS_ERR_INVALID_ARG;
+  return ds::launch_confidence(logits, dtype, rows, V, ld, row_list, n_listed, conf, tok, workspace,
+                               workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int ds_unmask_select(const ds_select_params *p, void *stream) {
+  if (!p) return DS_ERR_INVALID_ARG;
+  if (p->B < 0 || p->K < 1 || p->K > 4096 || p->ratio_extra < 0) return DS_ERR_INVALID_ARG;
+  if (!(p->tau0 == p->tau0) || !(p->alpha == p->alpha) || !(p->eos_tau == p->eos_tau)) return DS_ERR_INVALID_ARG;
+  if (!p->active_cnt) return DS_ERR_INVALID_ARG;
+  if (p->B > 0 && (!p->conf || !p->tok || !p->masked || !p->x_block || !p->sel_idx || !p->sel_cnt ||
+                   !p->block_done || !p->eos_exit || !p->active_seq))
+    return DS_ERR_INVALID_ARG;
+  if (p->seq_list && (p->n_seq < 0 || p->n_seq > p->B)) return DS_ERR_INVALID_ARG;
+  if (!p->seq_list && p->n_seq_dev) return DS_ERR_INVALID_ARG;
+  return ds::launch_select(*p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int ds_read_status(const uint32_t *device_status, void *stream, uint32_t *host_out) {
+  if (!device_status || !host_out) return DS_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  DS_CUDA_OK(cudaMemcpyAsync(host_out, device_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+  DS_CUDA_OK(cudaStreamSynchronize(st));
+  return DS_OK;
+}
+
+const char *ds_strerror(int code) {
+  switch (code) {
+    case DS_OK: return "ok";
+    case DS_ERR_INVALID_ARG: return "invalid argument";
+    case DS_ERR_UNSUPPORTED: return "shape or type outside the kernels' envelope";
+    case DS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case DS_ERR_CUDA: return "CUDA call failed";
+    default: return "unknown status";
+  }
+}
+
+int ds_version(void) { return 1000; }
+
+int64_t ds_launch_count(void) { return ds::g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,51 @@
+// Shared host/device helpers of the sm_100a denoising-step library.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ds.h"
+
+namespace ds {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Count of kernels launched through the C ABI (read by ds_launch_count()).
+void note_launch(int n = 1);
+
+inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+// Number of SMs of the current device (cached per device).
+int sm_count();
+
+#define DS_CUDA_OK(expr)                          \
+  do {                                            \
+    cudaError_t _e = (expr);                      \
+    if (_e != cudaSuccess) {                      \
+      (void)cudaGetLastError();                   \
+      return DS_ERR_CUDA;                         \
+    }                                             \
+  } while (0)
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ float bf16lo_to_f32(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi_to_f32(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Launchers implemented in the per-kernel translation units.
+int launch_confidence(const void *logits, int dtype, int64_t rows, int64_t V, int64_t ld,
+                      const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
+                      void *workspace, size_t workspace_bytes, cudaStream_t stream);
+size_t confidence_workspace_bytes(int64_t rows, int64_t V, int dtype);
+int launch_select(const ds_select_params &p, cudaStream_t stream);
+int launch_attn_simt(const ds_attn_params &p, cudaStream_t stream);
+int launch_attn_tc(const ds_attn_params &p, cudaStream_t stream);
+bool attn_tc_supported(const ds_attn_params &p);
+size_t attn_tc_workspace_bytes(const ds_attn_params &p);
+
+}  // namespace ds

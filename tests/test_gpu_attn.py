@@ -1,0 +1,208 @@
+"""GPU parity of ds_attn_pruned (Eq. 7-8) against the CPU oracle, through the C ABI.
+
+Bar: max-abs error <= 1e-2 on unit-scale values.  With N(0,1) inputs the
+outputs are small (softmax is diffuse), so the error is also bounded relative
+to the RMS of the reference output, and a "peaked" case (queries x4) gives
+unit-scale outputs.  Small cases are compared element by element; the full
+size configurations on sampled (batch, head) slices and sampled query rows,
+which the oracle computes one by one from the same device-generated data."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2601_17917_b200 as ds
+from paper_2601_17917_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+ABS_BAR = 1e-2
+
+
+def _tol(dtype):
+    # own bounds: fp32 path ~1e-5; bf16 path = output rounding (2^-9 relative) + bf16 probabilities
+    return (2e-5, 1e-4) if dtype == torch.float32 else (4e-3, 2e-2)
+
+
+def _np(t):
+    return t.float().cpu().numpy()
+
+
+def _compare(out, ref, dtype, what=""):
+    out = _np(out).astype(np.float64)
+    err = np.abs(out - ref).max()
+    rms = math.sqrt(float((ref ** 2).mean())) + 1e-30
+    own_abs, own_rel = _tol(dtype)
+    assert np.isfinite(out).all(), what
+    assert err <= ABS_BAR, (what, err)
+    assert err <= own_abs + own_rel * max(rms, np.abs(ref).max()), (what, err, rms)
+    return err, rms
+
+
+def _run_small(B, Hq, Hkv, D, P, T, idx, dtype, seed=0, q_scale=1.0, want_lse=True, noncontig=False):
+    cfg = wl.StepConfig("t", B=B, Hq=Hq, Hkv=Hkv, D=D, P=P, gen=T, K=1, w=0, keep_last=False,
+                        dtype="f32" if dtype == torch.float32 else "bf16", V=8, spike_p=0, seed=seed)
+    x = wl.attention_inputs(cfg, device=DEV, q_scale=q_scale)
+    if noncontig:   # strided views: padded rows and a head-major parent
+        for k in list(x):
+            t = x[k]
+            big = torch.zeros(t.shape[0], t.shape[2], t.shape[1], t.shape[3] + 16, dtype=t.dtype, device=DEV)
+            big[..., : t.shape[3]] = t.transpose(1, 2)
+            x[k] = big.transpose(1, 2)[..., : t.shape[3]]
+    idx_t = torch.as_tensor(np.asarray(idx), dtype=torch.int32, device=DEV)
+    Lq = idx_t.shape[-1]
+    lse = torch.empty((B, Hq, Lq), dtype=torch.float32, device=DEV) if want_lse else None
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    scale = 1.0 / math.sqrt(D)
+    kp, vp = (x["k_pre"], x["v_pre"]) if P > 0 else (None, None)
+    out = ds.ds_attn_pruned(x["q_tail"], x["k_tail"], x["v_tail"], kp, vp, idx_t, scale, lse=lse, status=status)
+    torch.cuda.synchronize()
+    assert ds.ds_read_status(status) == 0
+    ref, ref_lse = oracle.attn(_np(x["q_tail"]), _np(x["k_tail"]), _np(x["v_tail"]), _np(x["k_pre"]),
+                               _np(x["v_pre"]), np.asarray(idx), scale, want_lse=True)
+    _compare(out, ref, dtype, f"B{B} Hq{Hq} Hkv{Hkv} D{D} P{P} T{T} Lq{Lq}")
+    if want_lse:
+        assert np.abs(_np(lse) - ref_lse).max() < (1e-4 if dtype == torch.float32 else 2e-2)
+    return out
+
+
+def test_tiny_config_fp32():
+    cfg = wl.CONFIGS["tiny"]
+    idx = ds.retained_indices(cfg.gen, cfg.K, 0, cfg.w, cfg.keep_last)
+    assert len(idx) == 49
+    _run_small(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, cfg.P, cfg.T, idx, torch.float32, seed=cfg.seed)
+
+
+@pytest.mark.parametrize("Lq_spec", [1, 2, 33, 64, 65, 97, 128, 129, 130, 200, 257])
+@pytest.mark.parametrize("P", [0, 64, 100, 384, 1000])
+def test_bf16_tiles_and_ragged_tails(Lq_spec, P):
+    T = 300
+    # the paper's list shape: a contiguous run from row 0 plus the trailing position
+    idx = list(range(Lq_spec - 1)) + [T - 1] if Lq_spec > 1 else [T - 1]
+    _run_small(2, 2, 2, 128, P, T, idx, torch.bfloat16, seed=Lq_spec * 7 + P)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("G", [1, 4, 7])
+def test_gqa_head_grouping(D, G):
+    T = 160
+    idx = list(range(96)) + [T - 1]
+    _run_small(2, 2 * G, 2, D, 300, T, idx, torch.bfloat16, seed=D + G)
+
+
+def test_scattered_and_per_batch_index_lists():
+    rng = np.random.default_rng(3)
+    T, B = 500, 3
+    idx = np.stack([np.sort(rng.choice(T, 150, replace=False)) for _ in range(B)])
+    _run_small(B, 4, 2, 128, 200, T, idx, torch.bfloat16, seed=5)
+    _run_small(B, 4, 4, 64, 77, T, idx[:, :40], torch.float32, seed=6)
+    # runs that start on odd rows and have odd lengths
+    idx1 = list(range(3, 40)) + list(range(41, 46)) + list(range(100, 229)) + [499]
+    _run_small(1, 2, 2, 128, 130, T, idx1, torch.bfloat16, seed=7)
+
+
+def test_strided_inputs_and_no_lse():
+    idx = list(range(64)) + [199]
+    _run_small(2, 4, 2, 128, 256, 200, idx, torch.bfloat16, seed=9, noncontig=True, want_lse=False)
+    _run_small(1, 2, 2, 64, 50, 200, idx, torch.float32, seed=10, noncontig=True)
+
+
+def test_peaked_scores_unit_scale_outputs():
+    idx = list(range(128)) + [255]
+    out = _run_small(1, 4, 4, 128, 512, 256, idx, torch.bfloat16, seed=11, q_scale=4.0)
+    assert out.float().abs().max().item() > 0.5
+
+
+def test_all_retained_equals_unpruned_on_gpu():
+    """The structural identity on the GPU path itself: a window covering the whole suffix."""
+    cfg = wl.StepConfig("t", B=1, Hq=2, Hkv=2, D=128, P=128, gen=192, K=32, w=-1, keep_last=True,
+                        dtype="bf16", V=8, spike_p=0, seed=21)
+    x = wl.attention_inputs(cfg, device=DEV)
+    idx = ds.retained_indices(cfg.gen, cfg.K, 0, -1)
+    out = ds.ds_attn_pruned(x["q_tail"], x["k_tail"], x["v_tail"], x["k_pre"], x["v_pre"],
+                            torch.tensor(idx, dtype=torch.int32, device=DEV), 1 / math.sqrt(128))
+    ref = oracle.attn_full(_np(x["q_tail"]), _np(x["k_tail"]), _np(x["v_tail"]), _np(x["k_pre"]),
+                           _np(x["v_pre"]), 1 / math.sqrt(128))
+    _compare(out, ref, torch.bfloat16, "all retained")
+
+
+def test_out_of_range_index_sets_status_and_gpu_stays_healthy():
+    cfg = wl.StepConfig("t", B=1, Hq=2, Hkv=2, D=128, P=64, gen=100, K=32, w=0, keep_last=False,
+                        dtype="bf16", V=8, spike_p=0, seed=23)
+    x = wl.attention_inputs(cfg, device=DEV)
+    idx = torch.tensor([0, 1, 2, 1000], dtype=torch.int32, device=DEV)     # 1000 >= T: clamped to T-1
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = ds.ds_attn_pruned(x["q_tail"], x["k_tail"], x["v_tail"], x["k_pre"], x["v_pre"], idx, 0.1, status=status)
+    assert ds.ds_read_status(status) & ds.DS_DEV_INDEX
+    ref = oracle.attn(_np(x["q_tail"]), _np(x["k_tail"]), _np(x["v_tail"]), _np(x["k_pre"]), _np(x["v_pre"]),
+                      np.array([0, 1, 2, 99]), 0.1)
+    _compare(out, ref, torch.bfloat16, "clamped")
+    # errors reported by the host before any launch
+    with pytest.raises(ds.DsError) as e:
+        ds.ds_attn_pruned(x["q_tail"][..., :48], x["k_tail"][..., :48], x["v_tail"][..., :48],
+                          x["k_pre"][..., :48], x["v_pre"][..., :48], idx[:3], 0.1)
+    assert e.value.code in (ds.DS_ERR_UNSUPPORTED, ds.DS_ERR_INVALID_ARG)
+    torch.cuda.synchronize()
+
+
+# ---------------------------------------------------------------------------
+# full-size configurations, sampled
+# ---------------------------------------------------------------------------
+def _sampled_parity(cfg, n_slices=8, q_rows=None, layer=0, seed=0):
+    x = wl.attention_inputs(cfg, device=DEV, layer=layer)
+    idx = ds.retained_indices(cfg.gen, cfg.K, 0, cfg.w, cfg.keep_last)
+    idx_t = torch.tensor(idx, dtype=torch.int32, device=DEV)
+    scale = 1.0 / math.sqrt(cfg.D)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = ds.ds_attn_pruned(x["q_tail"], x["k_tail"], x["v_tail"], x["k_pre"], x["v_pre"], idx_t, scale,
+                            status=status)
+    torch.cuda.synchronize()
+    assert ds.ds_read_status(status) == 0
+    assert torch.isfinite(out.float()).all()
+    rng = np.random.default_rng(seed)
+    pairs = {(0, 0), (cfg.B - 1, cfg.Hq - 1), (0, cfg.Hq - 1), (cfg.B - 1, 0)}
+    while len(pairs) < min(n_slices, cfg.B * cfg.Hq):
+        pairs.add((int(rng.integers(cfg.B)), int(rng.integers(cfg.Hq))))
+    G = cfg.Hq // cfg.Hkv
+    ia = np.asarray(idx)
+    worst = 0.0
+    for b, h in sorted(pairs):
+        g = h // G
+        sl = lambda t, hh: _np(t[b:b + 1, hh:hh + 1])
+        q, kt, vt = sl(x["q_tail"], h), sl(x["k_tail"], g), sl(x["v_tail"], g)
+        kp, vp = sl(x["k_pre"], g), sl(x["v_pre"], g)
+        if q_rows is None:
+            ref = oracle.attn(q, kt, vt, kp, vp, ia, scale)[0, 0]
+            got = out[b, h]
+        else:
+            # sampled query rows: softmax attention does not depend on key order, so the keys of the
+            # retained rows that are not sampled are handed to the oracle as extra prefix rows
+            pick = np.sort(rng.choice(len(idx), q_rows, replace=False))
+            pick[0], pick[-1] = 0, len(idx) - 1
+            pick = np.unique(pick)
+            rest = np.setdiff1d(np.arange(len(idx)), pick)
+            kp2 = np.concatenate([kp, kt[:, :, ia[rest]]], 2)
+            vp2 = np.concatenate([vp, vt[:, :, ia[rest]]], 2)
+            ref = oracle.attn(q, kt, vt, kp2, vp2, ia[pick], scale)[0, 0]
+            got = out[b, h][torch.as_tensor(pick, device=DEV)]
+        err, _ = _compare(got, ref, x["q_tail"].dtype, f"{cfg.name} b{b} h{h}")
+        worst = max(worst, err)
+    return worst
+
+
+@pytest.mark.parametrize("name", ["llada1", "dream16", "long32-w0", "long32-w64", "long32-w256"])
+def test_full_size_configs_sampled(name):
+    _sampled_parity(wl.CONFIGS[name], n_slices=8)
+
+
+def test_full_size_llada_batched_layers():
+    cfg = wl.CONFIGS["llada8x32"]
+    for layer in (0, 13, 31):           # independent seeded caches; three of the 32 sampled
+        _sampled_parity(cfg, n_slices=6, layer=layer, seed=layer)
+
+
+def test_full_size_unpruned_reference_sampled_rows():
+    # "all 4032": the window covers the whole suffix; Lq = 4096, Lkv = 8192
+    _sampled_parity(wl.CONFIGS["long32-all"], n_slices=4, q_rows=16)
