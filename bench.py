@@ -142,8 +142,9 @@ class ClockSampler:
 class Step:
     """Device-resident inputs of one configuration and the three C-ABI calls of a step."""
 
-    def __init__(self, cfg, device, compact_tail=False):
+    def __init__(self, cfg, device, compact_tail=False, stages=("attn", "confidence", "select")):
         import torch
+        self.stages = tuple(stages)
         import paper_2601_17917_b200 as ds
         from paper_2601_17917_b200 import workloads as wl
         self.torch, self.ds, self.cfg, self.device = torch, ds, cfg, device
@@ -204,14 +205,17 @@ class Step:
         """One whole step.  ``events``: optional [4] CUDA events recorded between the stages."""
         if events:
             events[0].record()
-        for layer in range(self.cfg.n_layers):
-            self.attn(layer)
+        if "attn" in self.stages:
+            for layer in range(self.cfg.n_layers):
+                self.attn(layer)
         if events:
             events[1].record()
-        self.confidence()
+        if "confidence" in self.stages:
+            self.confidence()
         if events:
             events[2].record()
-        self.select()
+        if "select" in self.stages:
+            self.select()
         if events:
             events[3].record()
 
@@ -378,6 +382,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stages", default="attn,confidence,select",
+                    help="comma list of the stages a step runs (profiling a single kernel)")
     args = ap.parse_args()
 
     from paper_2601_17917_b200 import workloads as wl
@@ -408,7 +414,7 @@ def main():
     warmup = max(args.warmup, 3)
     # replicas: every rank draws its own batch (its rank offsets the seed); no data-path collective
     rcfg = wl.shrink(cfg, seed=cfg.seed + 100000 * rank)
-    step = Step(rcfg, device)
+    step = Step(rcfg, device, stages=args.stages.split(","))
     sampler = ClockSampler(local)
     sampler.start()
     total_ms, stage_ms, launches, windows, extra = time_resident(step, args.steps, warmup, sampler, barrier)
@@ -425,7 +431,7 @@ def main():
     value = world * 1e3 / ms_per_step
 
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.stages == "attn,confidence,select":
         e2e_steps = max(3, min(args.steps, 20))
         del step.layers[1:]
         torch.cuda.empty_cache()
@@ -475,11 +481,18 @@ def main():
                                 "algorithmic_bytes": c_bytes},
         "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
     }
+    if args.stages != "attn,confidence,select":
+        line["stages"] = args.stages          # partial step: a profiling run, not a bench value
     if e2e:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
-        smp = OracleSample(cfg, 64, 512)
+        smp = OracleSample(cfg, 32, 128)
         full_s, spent = smp.time()
+        # grow the sample towards ~10 s of CPU work (never beyond the whole workload)
+        grow = max(1.0, min(10.0 / max(spent, 1e-3), 64.0))
+        if grow > 1.5:
+            smp = OracleSample(cfg, int(32 * grow), int(128 * grow))
+            full_s, spent = smp.time()
         line["cpu_baseline"] = {"value": 1.0 / full_s, "unit": "steps/s", "cores": smp.cores, "kind": "oracle",
                                 "sample": smp.sample, "sample_seconds": spent}
     print(json.dumps(line), flush=True)
