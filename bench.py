@@ -384,10 +384,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--stages", default="attn,confidence,select",
                     help="comma list of the stages a step runs (profiling a single kernel)")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the batch size of the configuration (small cases for profiler captures)")
     args = ap.parse_args()
 
     from paper_2601_17917_b200 import workloads as wl
     cfg = wl.CONFIGS[args.config]
+    if args.batch > 0:
+        cfg = wl.shrink(cfg, B=args.batch, name=f"{cfg.name}-B{args.batch}")
     if args.impl == "reference":
         run_reference(args, cfg)
         return
