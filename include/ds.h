@@ -51,7 +51,8 @@ typedef enum {
   DS_ERR_INVALID_ARG = 1, /* null pointer, negative size, inconsistent shape, misaligned pointer/stride */
   DS_ERR_UNSUPPORTED = 2, /* well-formed request outside the kernels' envelope */
   DS_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or smaller than the *_workspace() query */
-  DS_ERR_CUDA = 4         /* a CUDA runtime/driver call failed (launch, tensor-map encode, ...) */
+  DS_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (launch, tensor-map encode, ...) */
+  DS_ERR_STATIC_LIMIT = 5 /* ds_confidence_static only: more rows than its fixed scratch can serve */
 } ds_status;
 
 /* bits OR-ed into the optional device status word */
@@ -141,6 +142,44 @@ DS_API size_t ds_confidence_workspace(int64_t rows, int64_t V, int32_t dtype);
 DS_API int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_t V, int64_t ld,
                   const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
                   void *workspace, size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------
+ * ds_confidence_static  (no counterpart in the paper: a packaging variant)
+ *
+ * The same computation and the same kernel as ds_confidence, for callers that
+ * have no way to hand over a workspace because they may not allocate device
+ * memory at the point of the call: code running inside another framework's
+ * memory plan, a plugin whose host forbids cudaMalloc after start-up, a
+ * real-time loop that must not touch the allocator.  The scratch the split-row
+ * reduction needs (one ticket per processed row plus the partial results)
+ * lives instead in a fixed array inside the library's device image:
+ * 4 * MAX_ROWS + 32 * MAX_ROWS bytes = 144 KiB, held by every GPU that loads
+ * the library until the process exits.
+ *
+ * Arguments as for ds_confidence, minus the workspace.  This function and
+ * everything it calls allocate and free nothing, on the host or the device.
+ *
+ * Limits and errors: at most DS_CONFIDENCE_STATIC_MAX_ROWS processed rows
+ * (`rows`, or `n_listed` with a row list); more returns DS_ERR_STATIC_LIMIT
+ * and launches nothing.  The other argument errors are those of
+ * ds_confidence.
+ *
+ * First call on a device: it looks up the device address of the scratch array
+ * (a CUDA runtime query, remembered per device; the device that is current at
+ * the call is the one set up).  Make that first call outside any stream
+ * capture.
+ *
+ * Sharing: every call on a device uses the same array, and the array keeps
+ * the previous call's contents; the function clears the tickets it is about
+ * to use on `stream` before the kernel.  Two calls that can overlap on the GPU
+ * (different streams without an ordering between them) race on the array and
+ * give wrong results: order them, or use ds_confidence with separate
+ * workspaces.
+ * ------------------------------------------------------------------------ */
+#define DS_CONFIDENCE_STATIC_MAX_ROWS 4096
+DS_API int ds_confidence_static(const void *logits, int32_t dtype, int64_t rows, int64_t V, int64_t ld,
+                         const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
+                         void *stream);
 
 /* ------------------------------------------------------------------------
  * ds_unmask_select  (Eq. 9, Eq. 10, Eq. 5, block termination, early exit)

@@ -18,12 +18,13 @@ from . import workloads  # noqa: F401  (seeded synthetic inputs)
 
 __all__ = [
     "lib", "retained_indices", "ds_attn_pruned", "ds_attn_pruned_workspace", "ds_confidence",
-    "ds_confidence_workspace", "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
+    "ds_confidence_workspace", "ds_confidence_static", "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
     "ds_launch_count", "DsError", "DS_F32", "DS_BF16", "DS_DEV_INDEX", "DS_DEV_TIMEOUT",
 ]
 
 DS_F32, DS_BF16 = 0, 1
-DS_OK, DS_ERR_INVALID_ARG, DS_ERR_UNSUPPORTED, DS_ERR_WORKSPACE, DS_ERR_CUDA = range(5)
+DS_OK, DS_ERR_INVALID_ARG, DS_ERR_UNSUPPORTED, DS_ERR_WORKSPACE, DS_ERR_CUDA, DS_ERR_STATIC_LIMIT = range(6)
+DS_CONFIDENCE_STATIC_MAX_ROWS = 4096
 DS_DEV_INDEX, DS_DEV_TIMEOUT = 1, 2
 
 _LIB_PATH = Path(__file__).resolve().parent / "libds_b200.so"
@@ -80,6 +81,10 @@ def lib() -> ctypes.CDLL:
         L.ds_confidence.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.ds_confidence_static.restype = ctypes.c_int
+        L.ds_confidence_static.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                           ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                                           ctypes.c_void_p, ctypes.c_void_p]
         L.ds_unmask_select.restype = ctypes.c_int
         L.ds_unmask_select.argtypes = [ctypes.POINTER(_SelectParams), ctypes.c_void_p]
         L.ds_read_status.restype = ctypes.c_int
@@ -230,6 +235,28 @@ def ds_confidence(logits, row_list=None, conf=None, tok=None, workspace=None, st
                              _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
     if rc != DS_OK:
         raise DsError(rc, "ds_confidence")
+    return conf, tok
+
+
+def ds_confidence_static(logits, conf, tok, row_list=None, stream=None):
+    """Eq. 4 like ``ds_confidence``, through the entry point that needs no workspace: its scratch is a
+    fixed array inside the library, so the call itself allocates nothing.  For callers that cannot
+    allocate device memory where they call from.  ``conf`` f32 [rows] and ``tok`` i32 [rows] must be
+    passed in (this wrapper creates no tensor either).  At most DS_CONFIDENCE_STATIC_MAX_ROWS rows are
+    processed per call; calls that may overlap on the GPU must be ordered, they share the scratch."""
+    _check_dev(logits, row_list, conf, tok)
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits must be [rows, V] with contiguous rows")
+    rows, V = logits.shape
+    if conf.dtype != torch.float32 or tok.dtype != torch.int32 or conf.numel() < rows or tok.numel() < rows:
+        raise ValueError("conf must be f32 [rows] and tok i32 [rows]")
+    if row_list is not None and row_list.dtype != torch.int32:
+        raise TypeError("row_list must be int32")
+    rc = lib().ds_confidence_static(_ptr(logits), _dtype_code(logits), rows, V, logits.stride(0), _ptr(row_list),
+                                    0 if row_list is None else row_list.numel(), _ptr(conf), _ptr(tok),
+                                    _stream(stream))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_confidence_static")
     return conf, tok
 
 

@@ -114,6 +114,19 @@ int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_t V, in
                                workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
+int ds_confidence_static(const void *logits, int32_t dtype, int64_t rows, int64_t V, int64_t ld,
+                         const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok, void *stream) {
+  if (dtype != DS_F32 && dtype != DS_BF16) return DS_ERR_INVALID_ARG;
+  if (rows < 0 || V <= 0 || ld < V || V > 0x7fffffffLL) return DS_ERR_INVALID_ARG;
+  if (rows == 0) return DS_OK;
+  if (!logits || !conf || !tok) return DS_ERR_INVALID_ARG;
+  const size_t esz = dtype == DS_BF16 ? 2 : 4;
+  if (!ds::aligned(logits, esz) || !ds::aligned(conf, 4) || !ds::aligned(tok, 4)) return DS_ERR_INVALID_ARG;
+  if (row_list && (n_listed < 0 || n_listed > rows)) return DS_ERR_INVALID_ARG;
+  return ds::launch_confidence_static(logits, dtype, rows, V, ld, row_list, n_listed, conf, tok,
+                                      reinterpret_cast<cudaStream_t>(stream));
+}
+
 int ds_unmask_select(const ds_select_params *p, void *stream) {
   if (!p) return DS_ERR_INVALID_ARG;
   if (p->B < 0 || p->K < 1 || p->K > 4096 || p->ratio_extra < 0) return DS_ERR_INVALID_ARG;
@@ -142,6 +155,8 @@ const char *ds_strerror(int code) {
     case DS_ERR_UNSUPPORTED: return "shape or type outside the kernels' envelope";
     case DS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case DS_ERR_CUDA: return "CUDA call failed";
+    case DS_ERR_STATIC_LIMIT:
+      return "request exceeds the fixed scratch of the allocation-free entry point (too many rows)";
     default: return "unknown status";
   }
 }

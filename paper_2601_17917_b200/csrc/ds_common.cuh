@@ -42,6 +42,9 @@ int launch_confidence(const void *logits, int dtype, int64_t rows, int64_t V, in
                       const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
                       void *workspace, size_t workspace_bytes, cudaStream_t stream);
 size_t confidence_workspace_bytes(int64_t rows, int64_t V, int dtype);
+int launch_confidence_static(const void *logits, int dtype, int64_t rows, int64_t V, int64_t ld,
+                             const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
+                             cudaStream_t stream);
 int launch_select(const ds_select_params &p, cudaStream_t stream);
 int launch_attn_simt(const ds_attn_params &p, cudaStream_t stream);
 int launch_attn_tc(const ds_attn_params &p, cudaStream_t stream);

@@ -13,6 +13,7 @@
 // to the workspace; the CTA that arrives last (atomic ticket) merges them.
 #include <cfloat>
 #include <climits>
+#include <mutex>
 
 #include "ds_common.cuh"
 
@@ -254,7 +255,65 @@ inline int pick_splits(int64_t n_rows, int64_t V, int dtype) {
   return (int)want;
 }
 
+// Fixed scratch of ds_confidence_static: one ticket per processed row, then the partial triples.
+// It lives in every device that loads the library, for the life of the process.
+constexpr int kStaticRows = DS_CONFIDENCE_STATIC_MAX_ROWS;
+constexpr int kStaticPartials = 2 * kStaticRows;
+constexpr size_t kStaticTicketBytes = (size_t)kStaticRows * sizeof(unsigned);
+constexpr size_t kStaticBytes = kStaticTicketBytes + (size_t)kStaticPartials * sizeof(Triple);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void *g_static_ptr[kMaxDevices];  // device address of g_static_scratch, per device; null until set up
+
+// Device address of the scratch array on the current device.  In host code the array's name is only
+// a handle, so the address a kernel can use has to be asked for, once per device, with that
+// device current.
+int static_scratch(void **out) {
+  int dev = -1;
+  DS_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return DS_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void *ptr = nullptr;
+    DS_CUDA_OK(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    if (!ptr) return DS_ERR_CUDA;
+    g_static_ptr[dev] = ptr;
+  }
+  *out = g_static_ptr[dev];
+  return DS_OK;
+}
+
 }  // namespace
+
+int launch_confidence_static(const void *logits, int dtype, int64_t rows, int64_t V, int64_t ld,
+                             const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
+                             cudaStream_t stream) {
+  const int64_t n = row_list ? n_listed : rows;
+  if (n == 0) return DS_OK;
+  if (n > kStaticRows) return DS_ERR_STATIC_LIMIT;
+  const int splits = pick_splits(n, V, dtype);
+  if (n * splits > kStaticPartials) return DS_ERR_STATIC_LIMIT;
+  void *base = nullptr;
+  const int rc = static_scratch(&base);
+  if (rc != DS_OK) return rc;
+  unsigned *tickets = reinterpret_cast<unsigned *>(base);
+  Triple *partials = reinterpret_cast<Triple *>(reinterpret_cast<unsigned char *>(base) + kStaticTicketBytes);
+  // the array keeps whatever the previous call left: the tickets must start at zero
+  if (splits > 1) DS_CUDA_OK(cudaMemsetAsync(tickets, 0, (size_t)n * sizeof(unsigned), stream));
+  const dim3 grid((unsigned)(n * splits));
+  if (dtype == DS_BF16) {
+    confidence_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>(
+        reinterpret_cast<const __nv_bfloat16 *>(logits), V, ld, row_list, splits, conf, tok, partials, tickets);
+  } else {
+    confidence_kernel<float><<<grid, kThreads, 0, stream>>>(reinterpret_cast<const float *>(logits), V, ld,
+                                                           row_list, splits, conf, tok, partials, tickets);
+  }
+  DS_CUDA_OK(cudaGetLastError());
+  note_launch(1);
+  return DS_OK;
+}
 
 size_t confidence_workspace_bytes(int64_t rows, int64_t V, int dtype) {
   if (rows <= 0 || V <= 0) return 0;
