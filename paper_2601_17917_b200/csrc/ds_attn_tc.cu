@@ -5,26 +5,51 @@
 // M (row R = head_in_group * Lq + i), so every KV tile is read once per group.  KV is streamed as
 // 128-row tiles: first the cached prefix (tiled TMA boxes, out-of-range rows zero-filled), then the
 // retained tail rows named by the index list, fetched as 32-row TMA boxes where the list is
-// contiguous and as single-row boxes elsewhere.
+// contiguous and as single-row boxes elsewhere.  CTAs are persistent: CTA c takes items c, c + grid,
+// ... and the KV ring keeps streaming across item boundaries.
 //
-// Warp roles (192 threads, one CTA per SM):
-//   warps 0-3  softmax + epilogue; thread t owns TMEM lane t = S/O row t
-//   warp  4    TMA producer (lane 0 issues; the warp pre-loads the index list of each gathered tile)
-//   warp  5    TMEM allocation and MMA issue (lane 0)
-// Per KV tile j:  S[j%2] = Q K_j^T  (tcgen05.mma, both operands K-major, 128B swizzle)
-//                 softmax warps: tcgen05.ld S, running max with lazy rescale, P = 2^(s*c - m) as bf16
-//                 into a swizzled shared-memory tile
-//                 O += P V_j       (A = P K-major, B = V MN-major straight from its [kv][D] layout)
-// S is double buffered so Q K_{j+1}^T runs under the softmax of tile j.  The accumulator O is only
-// rescaled when a row maximum grows by more than 2^8 (the stale maximum keeps P within bf16/fp32
-// range), which removes the TMEM round trip from the steady state.
+// "Extra" rows.  The retained set is block + window + the trailing position, so the stacked row
+// count is often 128 m + 1.  Up to 8 rows beyond the last full M-tile do not get a tile of their own:
+// they ride along with that tile as a second, transposed problem  S_x^T = K Q_x^T  (M = 128 keys,
+// N = 16) and  O_x^T = V^T P_x^T  (M = D, N = 16), which costs a fraction of a full tile on the
+// tensor cores.  There the keys lie along TMEM lanes, so a column maximum would need a cross-lane
+// reduction per tile; instead those columns are expressed against a reference exponent that is only
+// moved (with an exact rescale) when a score exceeds it by more than 2^24.
 //
-// Every mbarrier wait is bounded; on expiry the thread raises DS_DEV_TIMEOUT in the status word,
-// all roles leave their loops, outstanding TMA copies are waited for (bounded), TMEM is freed and the
-// CTA returns.
+// Warp roles (480 threads, one CTA per SM):
+//   warps 0-7  softmax + epilogue.  Warp w works on the 16 TMEM lanes 32 (w % 4) + 16 (w / 4) ..;
+//              two threads share a row (lanes l and l + 16 of the warp take the two column halves of
+//              every S tile, tcgen05.ld shape 16x32bx2), so a row maximum is one shuffle away and
+//              every scheduler has two softmax warps.
+//   warp  8    TMA producer (lane 0 issues; the warp stages the index list of each gathered tile)
+//   warp  9    TMEM allocation; issues Q K^T (one elected lane)
+//   warps 10-13 softmax + epilogue of the transposed problem (thread = key of the tile; idle in items
+//              without extra rows), kept apart so that its cross-warp agreement never sits on the
+//              main rows' critical path
+//   warp 14    issues P V.  Issuing blocks while the tensor pipe's queue is full, so the two streams
+//              have an issuer each; the one dependency the pipe no longer orders by itself (Q K^T of
+//              tile g + 2 overwrites the buffer P V of tile g reads) is an explicit barrier wait.
+// Per KV tile:  S[g%2] = Q K^T            (tcgen05.mma, both operands K-major in shared memory)
+//               softmax warps: tcgen05.ld S, row maximum, P = 2^(s*c - m) as bf16 written over the
+//               first 64 columns of the same S buffer
+//               O += P V                   (A = P from TMEM, B = V MN-major straight from its [kv][D]
+//                                           layout)
+// S/P is double buffered so Q K^T of the next tile runs under the softmax of this one.  O is only
+// rescaled when a row maximum grows by more than 2^8 (the stale maximum keeps P within range), which
+// removes the TMEM round trip from the steady state.
+//
+// Barriers are mbarriers waited on by parity.  A parity wait can only tell two consecutive phases
+// apart, so every barrier here is arranged such that a waiter is never more than one phase behind
+// (barriers that could run ahead are double buffered by tile parity, and per-item barriers are
+// waited on by every participant at every item).
+//
+// Every wait is bounded (no hardware barrier inside the role loops); on expiry the thread raises
+// DS_DEV_TIMEOUT in the status word, all roles leave their loops, outstanding TMA copies are waited
+// for (bounded), TMEM is freed and the CTA returns.
 #include <cuda.h>
 
 #include <cstdio>
+#include <cstring>
 #include <mutex>
 
 #include "ds_common.cuh"
@@ -32,31 +57,61 @@
 namespace ds {
 namespace {
 
+// Optional timeline of CTA 0 (build with -DDS_TRACE): SM clock at a few points of every role's loop.
+#ifdef DS_TRACE
+__device__ long long g_trace[4][256][8];
+#define DS_TR(role, g, ev)                                              \
+  do {                                                                  \
+    if (blockIdx.x == 0 && (g) < 256) g_trace[role][g][ev] = clock64(); \
+  } while (0)
+#else
+#define DS_TR(role, g, ev) \
+  do {                     \
+  } while (0)
+#endif
+
 constexpr int kBlockM = 128;
 constexpr int kBlockN = 128;
-constexpr int kNumThreads = 192;
-constexpr int kChunkBytes = 128 * 128;  // one [128 rows][64 bf16] swizzled chunk
-constexpr int kPBytes = kBlockM * kBlockN * 2;
+constexpr int kSoftmaxWarps = 8;
+constexpr int kXWarps = 4;  // softmax of the transposed problem (one per TMEM lane quadrant)
+constexpr int kNumThreads = (kSoftmaxWarps + 3 + kXWarps) * 32;
+constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1, kXWarp0 = kSoftmaxWarps + 2;
+constexpr int kPvWarp = kXWarp0 + kXWarps;  // second MMA issuer
+constexpr int kChunkBytes = 128 * 128;      // one [128 rows][64 bf16] swizzled chunk
+constexpr int kXRows = 16;                  // N of the transposed problem (the smallest N for M = 128)
+constexpr int kXMax = 8;                    // extra rows actually served
+constexpr int kXChunkBytes = kXRows * 128;
+constexpr int kIdxCap = 2048;               // entries of a shared index list kept in shared memory
 constexpr uint32_t kSpinLimit = 1u << 20;
-constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr float kRescaleThreshold = 8.0f;   // log2 units
+constexpr float kXLimit = 24.0f;            // log2 units a transposed score may exceed its reference by
 
 template <int D>
 struct Geo {
-  static constexpr int kChunks = D / 64;                     // 64-column chunks per tile
-  static constexpr int kTileBytes = kChunks * kChunkBytes;   // Q / K / V tile
-  static constexpr int kSlots = (D == 128) ? 5 : 10;         // ring of K/V tiles
+  static constexpr int kChunks = D / 64;                    // 64-column chunks per tile
+  static constexpr int kTileBytes = kChunks * kChunkBytes;  // Q / K / V tile
+  static constexpr int kSlots = (D == 128) ? 5 : 10;        // ring of K/V tiles
   static constexpr int kOffQ = 0;
-  static constexpr int kOffP = kTileBytes;
-  static constexpr int kOffRing = kOffP + kPBytes;
+  static constexpr int kOffQx = kTileBytes;                 // [kChunks][16 rows][128 B]
+  static constexpr int kOffPx = kOffQx + 2 * kXChunkBytes;  // [2 buffers][2 chunks][16 rows][128 B]
+  static constexpr int kOffRing = kOffPx + 4 * kXChunkBytes;
   static constexpr int kOffBar = kOffRing + kSlots * kTileBytes;
-  // barriers: q_full, s_full[2], s_free[2], p_full, pv_done, slot_full[kSlots], slot_empty[kSlots]
-  static constexpr int kNumBars = 7 + 2 * kSlots;
-  static constexpr int kOffIdx = kOffBar + 8 * kNumBars;     // int32[128] gathered-row indices
-  static constexpr int kOffMisc = kOffIdx + 4 * 128;         // tmem base, abort flag
+  // barriers: q_full, q_free, s_full[2], p_full[2], pv_done[2], o_free, xbar[2], ybar, o_full, px_full[2],
+  //           ox_free, sx_full[2], pvx_done[2], slot_full[kSlots], slot_empty[kSlots]
+  static constexpr int kNumBars = 20 + 2 * kSlots;
+  static constexpr int kOffIdx = kOffBar + 8 * kNumBars;     // int32[128] gathered-row indices of a KV tile
+  static constexpr int kOffIdxQ = kOffIdx + 4 * 128;         // int32[128] gathered-row indices of a query tile
+  static constexpr int kOffXflag = kOffIdxQ + 4 * 128;       // int[2 parity][4 warps]
+  static constexpr int kOffXcol = kOffXflag + 4 * 16;        // float[4 warps][8 columns]
+  static constexpr int kOffIdxCache = kOffXcol + 4 * 64;     // int32[kIdxCap] the index list, when all batches share it
+  static constexpr int kOffMisc = kOffIdxCache + 4 * kIdxCap;  // tmem base, abort flag
   static constexpr int kSmemBytes = kOffMisc + 16 + 1024;    // + slack to align the base to 1024
   static constexpr int kTmemCols = 512;
-  static constexpr int kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;
+  static constexpr int kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;  // P(g) overwrites columns 0..63 of S(g)
+  static constexpr int kTmemSx0 = 384, kTmemSx1 = 400, kTmemOx = 416;
 };
+static_assert(Geo<128>::kSmemBytes <= 227 * 1024, "shared memory budget");
+static_assert(Geo<64>::kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct TcParams {
   CUtensorMap kpre, vpre, k32, k1, v32, v1, q32, q1;
@@ -67,6 +122,9 @@ struct TcParams {
   float *lse;
   uint32_t *status;
   int B, Hq, Hkv, G, P, T, Lq;
+  int n_mtiles;      // M-tiles per (batch, KV head)
+  int x_rows;        // extra rows riding with the last M-tile (0 = none)
+  int n_items;       // B * Hkv * n_mtiles
   float scale_log2;  // softmax scale * log2(e)
 };
 
@@ -107,6 +165,33 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   *abort_flag = 1;
   return false;
 }
+// Bounded wait for two barriers at once (their polls overlap instead of adding up).
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b,
+                                           volatile int *abort_flag) {
+  bool a = false, b = false;
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (!a) a = mbar_try_wait(bar_a, parity_a);
+    if (!b) b = mbar_try_wait(bar_b, parity_b);
+    if (a && b) return true;
+    if (it > 128) {
+      __nanosleep(64);
+      if (*abort_flag) return false;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+// True in exactly one lane of the (converged) warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
@@ -130,8 +215,8 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 }
 
 // D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
@@ -139,33 +224,59 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// D[tmem] (+)= A[tmem] * B[smem]: A is M x 16, one row per lane, two bf16 per 32-bit column.
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // mbarrier arrives once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+// 16 lanes x 32 columns twice: threads 0-15 get columns taddr.., threads 16-31 the same 16 lanes at
+// columns taddr + kSplit...
+template <int kSplit>
+__device__ __forceinline__ void tmem_ld16x2_32(uint32_t taddr, uint32_t *r) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "tcgen05.ld.sync.aligned.16x32bx2.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32], %33;"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
+      : "r"(taddr), "n"(kSplit)
       : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+template <int kSplit>
+__device__ __forceinline__ void tmem_st16x2_32(uint32_t taddr, const uint32_t *r) {
   asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "tcgen05.st.sync.aligned.16x32bx2.x32.b32 [%32], %33, "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
       "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
       ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
         "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
         "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
-        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr), "n"(kSplit)
       : "memory");
+}
+// 32 lanes x 8 columns: thread t gets columns taddr .. taddr + 7 of lane t of the warp's quadrant.
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t *r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t *r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};" ::"r"(r[0]), "r"(r[1]),
+               "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(taddr)
+               : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -176,9 +287,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
          (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128.
-__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
-         ((uint32_t)(kBlockM >> 4) << 24);
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool a_mn_major, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -186,50 +297,81 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
 
 // ------------------------------------------------------------------------------------------------
-// Producer helper: fetch up to 128 gathered rows (logical rows R0 .. R0+n-1 of a stacked sequence whose
-// period is Lq) into a swizzled tile.  The whole warp calls it; lane 0 issues the copies.
-// Returns the bytes issued (valid on lane 0).
+// Producer helper: fetch n gathered rows (logical rows R0 .. R0+n-1 of a stacked sequence whose
+// period is Lq) into a swizzled tile whose 64-column chunks are chunk_stride bytes apart.  The whole
+// warp calls it; lane 0 issues the copies.  Returns the bytes issued (valid on lane 0).
 // ------------------------------------------------------------------------------------------------
 template <int D>
 __device__ __forceinline__ uint32_t gather_rows(const TcParams &prm, const CUtensorMap *map32, const CUtensorMap *map1,
-                                                uint32_t dst, uint32_t bar, int R0, int n, int head0, int b,
-                                                int32_t *idx_s, bool &bad_index) {
+                                                uint32_t dst, uint32_t chunk_stride, uint32_t bar, int R0, int n,
+                                                int head0, int b, int32_t *idx_s, const int32_t *idx_cache,
+                                                bool &bad_index, bool staged = false) {
   const int lane = threadIdx.x & 31;
-  const int32_t *ix = prm.idx + (long long)b * prm.idx_bstride;
-  __syncwarp();
-  for (int r = lane; r < n; r += 32) {
-    int v = ix[(R0 + r) % prm.Lq];
-    if (v < 0 || v >= prm.T) {
-      bad_index = true;
-      v = v < 0 ? 0 : prm.T - 1;
-    }
-    idx_s[r] = v;
+  const int Lq = prm.Lq;
+  // position of logical row R0 inside its head; divisions only when the stacking actually wraps
+  int head = head0, pos0 = R0;
+  if (pos0 >= Lq) {
+    head += pos0 / Lq;
+    pos0 %= Lq;
   }
   __syncwarp();
+  if (!staged) {  // otherwise idx_s already holds these rows (the K tile of the same rows came first)
+    const int32_t *ix = prm.idx + (long long)b * prm.idx_bstride;
+    for (int r = lane; r < n; r += 32) {
+      int pos = pos0 + r;
+      if (pos >= Lq) pos %= Lq;
+      int v;
+      if (idx_cache != nullptr && pos < kIdxCap) {
+        v = idx_cache[pos];  // validated when it was cached
+      } else {
+        v = ix[pos];
+        if (v < 0 || v >= prm.T) {
+          bad_index = true;
+          v = v < 0 ? 0 : prm.T - 1;
+        }
+      }
+      idx_s[r] = v;
+    }
+    __syncwarp();
+  }
   uint32_t bytes = 0;
   if (lane == 0) {
-    int r = 0;
+    int r = 0, pos = pos0;
     while (r < n) {
-      const int R = R0 + r;
-      const int head = head0 + R / prm.Lq;
       const int row = idx_s[r];
-      const bool box32 = ((r & 7) == 0) && (r + 32 <= n) && ((R % prm.Lq) + 32 <= prm.Lq) && (idx_s[r + 31] - row == 31);
-      if (box32) {
+      const bool box32 = ((r & 7) == 0) && (r + 32 <= n) && (pos + 32 <= Lq) && (idx_s[r + 31] - row == 31);
+      const int step = box32 ? 32 : 1;
 #pragma unroll
-        for (int c = 0; c < Geo<D>::kChunks; ++c) tma_load_4d(dst + c * kChunkBytes + r * 128, map32, bar, c * 64, row, head, b);
-        bytes += 32u * 128u * Geo<D>::kChunks;
-        r += 32;
-      } else {
-#pragma unroll
-        for (int c = 0; c < Geo<D>::kChunks; ++c) tma_load_4d(dst + c * kChunkBytes + r * 128, map1, bar, c * 64, row, head, b);
-        bytes += 128u * Geo<D>::kChunks;
-        r += 1;
+      for (int c = 0; c < Geo<D>::kChunks; ++c)
+        tma_load_4d(dst + c * chunk_stride + r * 128, box32 ? map32 : map1, bar, c * 64, row, head, b);
+      bytes += (uint32_t)step * 128u * Geo<D>::kChunks;
+      r += step;
+      pos += step;
+      if (pos >= Lq) {  // a 32-row box never crosses a head, so this is at most one wrap
+        pos -= Lq;
+        ++head;
       }
     }
   }
   return bytes;
+}
+
+struct Item {
+  int b, hk, mt, m_rows, x_rows;
+};
+__device__ __forceinline__ Item decode_item(const TcParams &prm, int item) {
+  Item it;
+  it.mt = item % prm.n_mtiles;
+  const int bh = item / prm.n_mtiles;
+  it.hk = bh % prm.Hkv;
+  it.b = bh / prm.Hkv;
+  const int rows_total = prm.G * prm.Lq;
+  it.x_rows = (it.mt == prm.n_mtiles - 1) ? prm.x_rows : 0;
+  it.m_rows = min(kBlockM, rows_total - it.x_rows - it.mt * kBlockM);
+  return it;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -245,31 +387,50 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
 
   const uint32_t bar0 = sbase + G_::kOffBar;
   const uint32_t bar_q_full = bar0;
-  const uint32_t bar_s_full = bar0 + 8;    // [2]
-  const uint32_t bar_s_free = bar0 + 24;   // [2]
-  const uint32_t bar_p_full = bar0 + 40;
-  const uint32_t bar_pv_done = bar0 + 48;
-  const uint32_t bar_slot_full = bar0 + 56;                       // [kSlots]
+  const uint32_t bar_q_free = bar0 + 8;
+  const uint32_t bar_s_full = bar0 + 16;     // [2]
+  const uint32_t bar_p_full = bar0 + 32;     // [2] a softmax warp may be one tile ahead of another
+  const uint32_t bar_pv_done = bar0 + 48;    // [2] by tile parity: a waiter may be two tiles behind the P V stream
+  const uint32_t bar_o_free = bar0 + 64;
+  const uint32_t bar_x = bar0 + 72;          // [2] transposed problem: "does this tile outgrow the reference" votes
+  const uint32_t bar_y = bar0 + 88;          // transposed problem: occasional exchanges (column maxima, sums)
+  const uint32_t bar_o_full = bar0 + 96;     // the last P V of an item has completed
+  const uint32_t bar_px_full = bar0 + 104;   // [2] P_x^T of a tile is in shared memory
+  const uint32_t bar_ox_free = bar0 + 120;   // the epilogue has read O_x^T
+  const uint32_t bar_sx_full = bar0 + 128;   // [2] S_x^T of a tile is in TMEM
+  const uint32_t bar_pvx_done = bar0 + 144;  // [2] O_x^T += V^T P_x^T of a tile has completed
+  const uint32_t bar_slot_full = bar0 + 160;                       // [kSlots]
   const uint32_t bar_slot_empty = bar_slot_full + 8 * G_::kSlots;  // [kSlots]
   int32_t *idx_s = reinterpret_cast<int32_t *>(smem + G_::kOffIdx);
+  int32_t *idxq_s = reinterpret_cast<int32_t *>(smem + G_::kOffIdxQ);
   volatile uint32_t *tmem_base_s = reinterpret_cast<volatile uint32_t *>(smem + G_::kOffMisc);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + G_::kOffMisc + 4);
 
-  const int mt = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
-  const int rows_total = prm.G * prm.Lq;                        // stacked query rows of this KV head
-  const int m_rows = min(kBlockM, rows_total - mt * kBlockM);   // valid rows of this M-tile
   const int n_pre = (prm.P + kBlockN - 1) / kBlockN;
   const int n_tail = (prm.Lq + kBlockN - 1) / kBlockN;
   const int n_tiles = n_pre + n_tail;
 
   if (tid == 0) {
     mbar_init(bar_q_full, 1);
+    mbar_init(bar_q_free, 1);
     mbar_init(bar_s_full, 1);
     mbar_init(bar_s_full + 8, 1);
-    mbar_init(bar_s_free, 4);
-    mbar_init(bar_s_free + 8, 4);
-    mbar_init(bar_p_full, 4);
+    mbar_init(bar_p_full, kSoftmaxWarps);
+    mbar_init(bar_p_full + 8, kSoftmaxWarps);
     mbar_init(bar_pv_done, 1);
+    mbar_init(bar_pv_done + 8, 1);
+    mbar_init(bar_o_free, kSoftmaxWarps);
+    mbar_init(bar_x, kXWarps);
+    mbar_init(bar_x + 8, kXWarps);
+    mbar_init(bar_y, kXWarps);
+    mbar_init(bar_o_full, 1);
+    mbar_init(bar_px_full, kXWarps);
+    mbar_init(bar_px_full + 8, kXWarps);
+    mbar_init(bar_ox_free, kXWarps);
+    mbar_init(bar_sx_full, 1);
+    mbar_init(bar_sx_full + 8, 1);
+    mbar_init(bar_pvx_done, 1);
+    mbar_init(bar_pvx_done + 8, 1);
     for (int s = 0; s < G_::kSlots; ++s) {
       mbar_init(bar_slot_full + 8 * s, 1);
       mbar_init(bar_slot_empty + 8 * s, 1);
@@ -277,230 +438,596 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     *abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 5) tmem_alloc(sbase + G_::kOffMisc, G_::kTmemCols);
+  if (warp == kMmaWarp) tmem_alloc(sbase + G_::kOffMisc, G_::kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_base_s;
   bool timed_out = false;
 
-  if (warp == 4) {
+  if (warp == kProducerWarp) {
     // ============================ TMA producer ============================
     bool bad_index = false;
-    {
-      const uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, sbase + G_::kOffQ, bar_q_full, mt * kBlockM, m_rows,
-                                            hk * prm.G, b, idx_s, bad_index);
-      if (lane == 0) mbar_arrive_expect_tx(bar_q_full, bytes);
-    }
-    int issued = 0;  // ring fills issued so far
-    for (int j = 0; j < n_tiles && !timed_out; ++j) {
-      for (int kv = 0; kv < 2; ++kv) {
-        const int slot = issued % G_::kSlots, use = issued / G_::kSlots;
-        const uint32_t dst = sbase + G_::kOffRing + slot * G_::kTileBytes;
-        const uint32_t full = bar_slot_full + 8 * slot;
-        bool ok = mbar_wait(bar_slot_empty + 8 * slot, (use & 1) ^ 1, abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) {
-          timed_out = true;
-          break;
-        }
-        if (j < n_pre) {
-          if (lane == 0) {
-            const CUtensorMap *map = kv ? &prm.vpre : &prm.kpre;
-#pragma unroll
-            for (int c = 0; c < G_::kChunks; ++c) tma_load_4d(dst + c * kChunkBytes, map, full, c * 64, j * kBlockN, hk, b);
-            mbar_arrive_expect_tx(full, G_::kTileBytes);
-          }
-        } else {
-          const int t0 = (j - n_pre) * kBlockN;
-          const int n = min(kBlockN, prm.Lq - t0);
-          if (kv == 1 && n < kBlockN) {
-            // rows past the end of a V tile meet P = 0 in the MMA: make them zero, not stale
-            const int nz_rows = kBlockN - n;
-            for (int q = lane; q < nz_rows * 8 * G_::kChunks; q += 32) {
-              const int u = q % 8, row = n + (q / 8) % nz_rows, c = q / (8 * nz_rows);
-              *reinterpret_cast<uint4 *>(smem + G_::kOffRing + slot * G_::kTileBytes + c * kChunkBytes + row * 128 + u * 16) =
-                  make_uint4(0, 0, 0, 0);
-            }
-            fence_proxy_async();
-          }
-          const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, dst, full, t0, n, hk, b,
-                                                idx_s, bad_index);
-          if (lane == 0) mbar_arrive_expect_tx(full, bytes);
-        }
-        ++issued;
+    if (lane == 0) {
+      auto prefetch_map = [](const CUtensorMap *m) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
+      };
+      if (prm.P > 0) {
+        prefetch_map(&prm.kpre);
+        prefetch_map(&prm.vpre);
       }
+      prefetch_map(&prm.k32);
+      prefetch_map(&prm.k1);
+      prefetch_map(&prm.v32);
+      prefetch_map(&prm.v1);
+      prefetch_map(&prm.q32);
+      prefetch_map(&prm.q1);
+    }
+    // one index list for all batches: keep (the head of) it in shared memory, validated once
+    const int32_t *idx_cache = nullptr;
+    if (prm.idx_bstride == 0) {
+      int32_t *cache = reinterpret_cast<int32_t *>(smem + G_::kOffIdxCache);
+      for (int i = lane; i < min(prm.Lq, kIdxCap); i += 32) {
+        int v = prm.idx[i];
+        if (v < 0 || v >= prm.T) {
+          bad_index = true;
+          v = v < 0 ? 0 : prm.T - 1;
+        }
+        cache[i] = v;
+      }
+      __syncwarp();
+      idx_cache = cache;
+    }
+    const int n_my = (prm.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // items of this CTA
+    int q_next = 0;  // first item (in this CTA's order) whose query tile has not been requested yet
+    // Requests the query tile(s) of this CTA's kq-th item.  The caller has made sure the previous
+    // item's last Q K^T has completed.
+    auto issue_q = [&](int kq) {
+      const Item it = decode_item(prm, blockIdx.x + kq * gridDim.x);
+      uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
+                                      it.mt * kBlockM, it.m_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
+      if (it.x_rows > 0) {
+        // rows of the small query tile that are not loaded must be finite: clear the tile first
+        for (int q = lane; q < (2 * kXChunkBytes) / 16; q += 32)
+          *reinterpret_cast<uint4 *>(smem + G_::kOffQx + q * 16) = make_uint4(0, 0, 0, 0);
+        fence_proxy_async();
+        bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, sbase + G_::kOffQx, kXChunkBytes, bar_q_full,
+                                (it.mt + 1) * kBlockM, it.x_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
+      }
+      if (lane == 0) mbar_arrive_expect_tx(bar_q_full, bytes);
+    };
+    int issued = 0;  // ring fills issued so far
+    for (int k = 0; k < n_my && !timed_out; ++k) {
+      const Item it = decode_item(prm, blockIdx.x + k * gridDim.x);
+      for (int j = 0; j < n_tiles && !timed_out; ++j) {
+        for (int kv = 0; kv < 2; ++kv) {
+          const int slot = issued % G_::kSlots, use = issued / G_::kSlots;
+          const uint32_t dst = sbase + G_::kOffRing + slot * G_::kTileBytes;
+          const uint32_t full = bar_slot_full + 8 * slot;
+          DS_TR(0, issued >> 1, kv * 3 + 0);
+          // Wait for the ring slot.  The KV stream runs ahead of the query tiles across item
+          // boundaries, so while waiting, serve the query tile of the item these fills belong to as
+          // soon as the previous item has released the buffer.
+          bool got = false;
+          for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+            if (q_next <= k) {
+              bool ready = (q_next == 0) || mbar_try_wait(bar_q_free, (q_next - 1) & 1);
+              ready = __all_sync(0xffffffffu, ready);
+              if (ready) {
+                issue_q(q_next);
+                ++q_next;
+                continue;
+              }
+            }
+            bool e = mbar_try_wait(bar_slot_empty + 8 * slot, (use & 1) ^ 1);
+            e = __all_sync(0xffffffffu, e);
+            if (e) {
+              got = true;
+              break;
+            }
+            if (spin > 128) {
+              __nanosleep(64);
+              if (__any_sync(0xffffffffu, *abort_flag != 0)) break;
+            }
+          }
+          if (!got) {
+            *abort_flag = 1;
+            timed_out = true;
+            break;
+          }
+          DS_TR(0, issued >> 1, kv * 3 + 1);
+          if (j < n_pre) {
+            if (lane == 0) {
+              const CUtensorMap *map = kv ? &prm.vpre : &prm.kpre;
+#pragma unroll
+              for (int c = 0; c < G_::kChunks; ++c)
+                tma_load_4d(dst + c * kChunkBytes, map, full, c * 64, j * kBlockN, it.hk, it.b);
+              mbar_arrive_expect_tx(full, G_::kTileBytes);
+            }
+          } else {
+            const int t0 = (j - n_pre) * kBlockN;
+            const int n = min(kBlockN, prm.Lq - t0);
+            if (kv == 1 && n < kBlockN) {
+              // rows past the end of a V tile meet P = 0 in the MMA: make them zero, not stale
+              // (a row of a chunk is 8 x 16 bytes: 4 rows per pass of the warp)
+              uint8_t *tile = smem + G_::kOffRing + slot * G_::kTileBytes + (lane & 7) * 16;
+              for (int row = n + (lane >> 3); row < kBlockN; row += 4) {
+#pragma unroll
+                for (int c = 0; c < G_::kChunks; ++c)
+                  *reinterpret_cast<uint4 *>(tile + c * kChunkBytes + row * 128) = make_uint4(0, 0, 0, 0);
+              }
+              fence_proxy_async();
+            }
+            // the V fill of a tile directly follows its K fill: the staged row list is still valid
+            const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, dst, kChunkBytes,
+                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, bad_index, kv == 1);
+            if (lane == 0) mbar_arrive_expect_tx(full, bytes);
+          }
+          DS_TR(0, issued >> 1, kv * 3 + 2);
+          ++issued;
+        }
+      }
+    }
+    // query tiles whose KV fills all went out before their buffer was released
+    while (!timed_out && q_next < n_my) {
+      bool ok = (q_next == 0) || mbar_wait(bar_q_free, (q_next - 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) {
+        timed_out = true;
+        break;
+      }
+      issue_q(q_next);
+      ++q_next;
     }
     if (timed_out) {
       // let copies already in flight land before the CTA's shared memory goes away
-      for (int k = max(0, issued - G_::kSlots); k < issued; ++k)
-        for (uint32_t it = 0; it < 4096 && !mbar_try_wait(bar_slot_full + 8 * (k % G_::kSlots), (k / G_::kSlots) & 1); ++it)
+      for (int f = max(0, issued - G_::kSlots); f < issued; ++f)
+        for (uint32_t w = 0; w < 4096 && !mbar_try_wait(bar_slot_full + 8 * (f % G_::kSlots), (f / G_::kSlots) & 1); ++w)
           __nanosleep(256);
     }
     if (bad_index && prm.status) atomicOr(prm.status, DS_DEV_INDEX);
-  } else if (warp == 5) {
-    // ============================ MMA issuer ============================
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = instr_desc(kBlockN, false);
-      constexpr uint32_t idesc_pv = instr_desc(D, true);
-      const uint32_t q_addr = sbase + G_::kOffQ, p_addr = sbase + G_::kOffP;
-      auto issue_qk = [&](int j) -> bool {
-        const int fill = 2 * j, slot = fill % G_::kSlots, use = fill / G_::kSlots;
-        if (!mbar_wait(bar_slot_full + 8 * slot, use & 1, abort_flag)) return false;
-        if (!mbar_wait(bar_s_free + 8 * (j & 1), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
-        tc_fence_after();
-        const uint32_t k_addr = sbase + G_::kOffRing + slot * G_::kTileBytes;
-        const uint32_t d = tmem + ((j & 1) ? G_::kTmemS1 : G_::kTmemS0);
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = (ks / 4) * kChunkBytes + (ks % 4) * 32;
-          umma_bf16(d, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_qk, ks > 0);
-        }
-        umma_commit(bar_s_full + 8 * (j & 1));
-        umma_commit(bar_slot_empty + 8 * slot);
-        return true;
-      };
-      bool ok = mbar_wait(bar_q_full, 0, abort_flag);
-      if (ok) ok = issue_qk(0);
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        if (j + 1 < n_tiles) ok = issue_qk(j + 1);
-        if (!ok) break;
-        const int fill = 2 * j + 1, slot = fill % G_::kSlots, use = fill / G_::kSlots;
-        if (!mbar_wait(bar_slot_full + 8 * slot, use & 1, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(bar_p_full, j & 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t v_addr = sbase + G_::kOffRing + slot * G_::kTileBytes;
-#pragma unroll
-        for (int ks = 0; ks < kBlockN / 16; ++ks) {
-          const uint64_t a = smem_desc(p_addr + (ks / 4) * kChunkBytes + (ks % 4) * 32, 16, 1024);
-          const uint64_t bdesc = smem_desc(v_addr + ks * 2048, kChunkBytes, 1024);
-          umma_bf16(tmem + G_::kTmemO, a, bdesc, idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
-        }
-        umma_commit(bar_pv_done);
-        umma_commit(bar_slot_empty + 8 * slot);
-      }
-      timed_out = !ok;
-    }
-  } else {
-    // ============================ softmax + epilogue ============================
-    const int row = tid;                                  // TMEM lane = row of the M-tile
-    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-    float m_used = -INFINITY;                             // maximum the probabilities are expressed against (log2 units)
-    float l_sum = 0.f;
-    const float c2 = prm.scale_log2;
-    uint8_t *p_row = smem + G_::kOffP + row * 128;
+  } else if (warp == kMmaWarp) {
+    // ============================ MMA issuer: S = Q K^T ============================
+    // The whole warp walks the loop (uniform control flow keeps descriptors in uniform registers);
+    // one elected lane issues the MMAs and commits.
+    constexpr uint32_t idesc_qk = instr_desc(kBlockN, false, false);
+    constexpr uint32_t idesc_qk_x = instr_desc(kXRows, false, false);  // S_x^T = K Q_x^T
+    const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+    // descriptors of byte 0 of each operand region; a K-step only adds to the address field
+    const uint64_t dq = smem_desc(sbase + G_::kOffQ, 16, 1024);
+    const uint64_t dqx = smem_desc(sbase + G_::kOffQx, 16, 1024);
+    const uint64_t dk0 = smem_desc(sbase + G_::kOffRing, 16, 1024);  // K tile, K-major
     bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
-      ok = mbar_wait(bar_s_full + 8 * (j & 1), (j >> 1) & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
+    int g0 = 0;   // tiles processed by this CTA before the current item
+    int k = 0;
+    int gx0 = 0;  // tiles of items with extra rows before the current item
+    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
+      const bool has_x = (D == 128) && decode_item(prm, item).x_rows > 0;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full, k & 1, abort_flag));
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int g = g0 + j, gx = gx0 + j;
+        const int fill = 2 * g, slot = fill % G_::kSlots, use = fill / G_::kSlots;
+        // the K tile has landed, and S[g % 2] is free: P V of tile g - 2, the reader of the P it still
+        // holds, has completed
+        bool w;
+        if (g >= 2)
+          w = mbar_wait2(bar_slot_full + 8 * slot, use & 1, bar_pv_done + 8 * (g & 1), ((g - 2) >> 1) & 1, abort_flag);
+        else
+          w = mbar_wait(bar_slot_full + 8 * slot, use & 1, abort_flag);
+        if (!__all_sync(0xffffffffu, w)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint64_t dk = dk0 + (uint64_t)((slot * G_::kTileBytes) >> 4);
+        if (elect_one()) {
+          DS_TR(1, g, 0);
+          const uint32_t d = tm + ((g & 1) ? G_::kTmemS1 : G_::kTmemS0);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t off = ((ks / 4) * kChunkBytes + (ks % 4) * 32) >> 4;
+            umma_ss(d, dq + off, dk + off, idesc_qk, ks > 0);
+          }
+          umma_commit(bar_s_full + 8 * (g & 1));
+        }
+        __syncwarp();
+        if (has_x && gx >= 2) {
+          // S_x^T and P_x^T buffers of this parity are free once the transposed P V of two such tiles
+          // back has completed (which also means its softmax warps have moved on)
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_pvx_done + 8 * (gx & 1), ((gx - 2) >> 1) & 1, abort_flag))) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+        }
+        if (elect_one()) {
+          if (has_x) {
+            const uint32_t dx = tm + ((gx & 1) ? G_::kTmemSx1 : G_::kTmemSx0);  // buffers by x-tile parity
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+              const uint32_t off = ((ks / 4) * kChunkBytes + (ks % 4) * 32) >> 4;
+              const uint32_t offx = ((ks / 4) * kXChunkBytes + (ks % 4) * 32) >> 4;
+              umma_ss(dx, dk + off, dqx + offx, idesc_qk_x, ks > 0);
+            }
+            umma_commit(bar_sx_full + 8 * (gx & 1));
+          }
+          umma_commit(bar_slot_empty + 8 * slot);
+          if (j == n_tiles - 1) umma_commit(bar_q_free);
+          DS_TR(1, g, 1);
+        }
+        __syncwarp();
+      }
+      if (has_x) gx0 += n_tiles;
+    }
+    timed_out = !ok;
+  } else if (warp == kPvWarp) {
+    // ============================ MMA issuer: O += P V ============================
+    constexpr uint32_t idesc_pv = instr_desc(D, false, true);
+    constexpr uint32_t idesc_pv_x = instr_desc(kXRows, true, false);  // O_x^T = V^T P_x^T
+    const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+    const uint64_t dpx = smem_desc(sbase + G_::kOffPx, 16, 1024);
+    const uint64_t dv0 = smem_desc(sbase + G_::kOffRing, kChunkBytes, 1024);  // V tile, MN-major
+    bool ok = true;
+    int g0 = 0, k = 0;
+    int kx = 0;   // items with extra rows before the current one
+    int gx0 = 0;  // tiles of such items
+    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
+      const bool has_x = (D == 128) && decode_item(prm, item).x_rows > 0;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int g = g0 + j, gx = gx0 + j;
+        const int fill = 2 * g + 1, slot = fill % G_::kSlots, use = fill / G_::kSlots;
+        bool w = mbar_wait2(bar_slot_full + 8 * slot, use & 1, bar_p_full + 8 * (g & 1), (g >> 1) & 1, abort_flag);
+        // the epilogue of the previous item has read O before this item's first P V overwrites it
+        if (j == 0 && k > 0) w = w && mbar_wait(bar_o_free, (k - 1) & 1, abort_flag);
+        if (!__all_sync(0xffffffffu, w)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint64_t dv = dv0 + (uint64_t)((slot * G_::kTileBytes) >> 4);
+        if (elect_one()) {
+          DS_TR(1, g, 2);
+#pragma unroll
+          for (int ks = 0; ks < kBlockN / 16; ++ks)
+            umma_ts(tm + G_::kTmemO, tm + ((g & 1) ? G_::kTmemS1 : G_::kTmemS0) + ks * 8, dv + ((ks * 2048) >> 4),
+                    idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+          umma_commit(bar_pv_done + 8 * (g & 1));  // frees S[g % 2] for Q K^T of tile g + 2
+        }
+        __syncwarp();
+        if (has_x) {
+          // the transposed problem's probabilities come from their own warps
+          bool wx = mbar_wait(bar_px_full + 8 * (gx & 1), (gx >> 1) & 1, abort_flag);
+          if (j == 0 && kx > 0) wx = wx && mbar_wait(bar_ox_free, (kx - 1) & 1, abort_flag);
+          if (!__all_sync(0xffffffffu, wx)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+        }
+        if (elect_one()) {
+          if (has_x) {
+            if constexpr (D == 128) {
+#pragma unroll
+              for (int ks = 0; ks < kBlockN / 16; ++ks) {
+                const uint32_t offx = ((gx & 1) * 2 * kXChunkBytes + (ks / 4) * kXChunkBytes + (ks % 4) * 32) >> 4;
+                umma_ss(tm + G_::kTmemOx, dv + ((ks * 2048) >> 4), dpx + offx, idesc_pv_x, (j > 0 || ks > 0) ? 1u : 0u);
+              }
+              umma_commit(bar_pvx_done + 8 * (gx & 1));
+            }
+          }
+          umma_commit(bar_slot_empty + 8 * slot);
+          if (j == n_tiles - 1) umma_commit(bar_o_full);
+          DS_TR(1, g, 3);
+        }
+        __syncwarp();
+      }
+      if (has_x) {
+        ++kx;
+        gx0 += n_tiles;
+      }
+    }
+    timed_out = !ok;
+  } else if (warp >= kXWarp0 && warp < kXWarp0 + kXWarps) {
+    // ============================ transposed problem: softmax + epilogue ============================
+    // Thread = key `row` of the tile (TMEM lane of S_x^T) and, for O_x^T, head-dimension element `row`.
+    // The kXMax columns are the extra query rows.
+    const int xw = warp - kXWarp0;
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const float c2 = prm.scale_log2;
+    volatile int *xflag_s = reinterpret_cast<volatile int *>(smem + G_::kOffXflag);
+    volatile float *xcol_s = reinterpret_cast<volatile float *>(smem + G_::kOffXcol);
+    bool ok = true;
+    int g0 = 0, k = 0, gx0 = 0;
+    uint32_t n_y = 0;  // uses of bar_y so far (same in all four warps)
+    // exchange through bar_y: every warp has written its part, everyone may read after the wait
+    auto sync_y = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_y);
+      bool w = mbar_wait(bar_y, n_y & 1, abort_flag);
+      ++n_y;
+      return __all_sync(0xffffffffu, w);
+    };
+    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
+      const Item it = decode_item(prm, item);
+      if (!((D == 128) && it.x_rows > 0)) {
+        // nothing to do, but stay in step with the per-item barrier (a parity wait cannot skip phases)
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full, k & 1, abort_flag));
+        continue;
+      }
+      float mref[kXMax], lx[kXMax];
+#pragma unroll
+      for (int i = 0; i < kXMax; ++i) mref[i] = 0.f, lx[i] = 0.f;
+      for (int j = 0; j < n_tiles; ++j) {
+        const int gx = gx0 + j;
+        // S_x^T of this tile is ready (and with it the P_x^T buffer of this parity is free: the issuer
+        // waited for the transposed P V of two such tiles back)
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_sx_full + 8 * (gx & 1), (gx >> 1) & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t sx[kXMax];
+        tmem_ld8(lane_base + ((gx & 1) ? G_::kTmemSx1 : G_::kTmemSx0), sx);
+        tmem_wait_ld();
+        const int valid = (j < n_pre) ? min(kBlockN, prm.P - j * kBlockN) : min(kBlockN, prm.Lq - (j - n_pre) * kBlockN);
+        const bool kv_live = row < valid;  // keys past the end of a partial tile do not exist
+        // Exponents against the reference.  A tile that outgrows it (and the first tile, which has no
+        // reference yet) takes the slow path; the four warps vote.
+        float tx[kXMax];
+        bool over = (j == 0);
+#pragma unroll
+        for (int i = 0; i < kXMax; ++i) {
+          tx[i] = kv_live ? fmaf(__uint_as_float(sx[i]), c2, -mref[i]) : -INFINITY;
+          over = over || (tx[i] > kXLimit);
+        }
+        over = __any_sync(0xffffffffu, over);
+        if (lane == 0) {
+          xflag_s[(gx & 1) * 4 + xw] = over ? 1 : 0;
+          mbar_arrive(bar_x + 8 * (gx & 1));
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_x + 8 * (gx & 1), (gx >> 1) & 1, abort_flag));
+        if (!ok) break;
+        const bool x_slow = (xflag_s[(gx & 1) * 4 + 0] | xflag_s[(gx & 1) * 4 + 1] | xflag_s[(gx & 1) * 4 + 2] |
+                             xflag_s[(gx & 1) * 4 + 3]) != 0;
+        if (x_slow) {
+          // exact column maxima over the 128 keys of this tile
+          float cm[kXMax], fx[kXMax];
+#pragma unroll
+          for (int i = 0; i < kXMax; ++i) {
+            cm[i] = kv_live ? __uint_as_float(sx[i]) * c2 : -INFINITY;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cm[i] = fmaxf(cm[i], __shfl_xor_sync(0xffffffffu, cm[i], o));
+          }
+          if (lane == 0) {
+#pragma unroll
+            for (int i = 0; i < kXMax; ++i) xcol_s[xw * kXMax + i] = cm[i];
+          }
+          ok = sync_y();
+          if (!ok) break;
+#pragma unroll
+          for (int i = 0; i < kXMax; ++i) {
+            const float c = fmaxf(fmaxf(xcol_s[0 * kXMax + i], xcol_s[1 * kXMax + i]),
+                                  fmaxf(xcol_s[2 * kXMax + i], xcol_s[3 * kXMax + i]));
+            const float m_new = (j == 0) ? c : fmaxf(mref[i], c);
+            fx[i] = (j == 0) ? 0.f : ex2_approx(mref[i] - m_new);
+            lx[i] *= fx[i];
+            mref[i] = m_new;
+            tx[i] = kv_live ? fmaf(__uint_as_float(sx[i]), c2, -m_new) : -INFINITY;
+          }
+          // xcol_s is reused by the next exchange: nobody may still be reading it
+          ok = sync_y();
+          if (!ok) break;
+          if (j > 0) {
+            // O_x^T must be quiescent: the previous transposed P V has completed
+            ok = __all_sync(0xffffffffu,
+                            mbar_wait(bar_pvx_done + 8 * ((gx - 1) & 1), ((gx - 1) >> 1) & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t o[kXMax];
+            tmem_ld8(lane_base + G_::kTmemOx, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < kXMax; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * fx[i]);
+            tmem_st8(lane_base + G_::kTmemOx, o);
+            tmem_wait_st();
+          }
+        }
+        // P_x^T -> shared memory as a K-major [16 rows][128 keys] operand, 128-byte swizzle
+        uint8_t *pxb = smem + G_::kOffPx + (gx & 1) * 2 * kXChunkBytes + (row >> 6) * kXChunkBytes + (row & 7) * 2;
+        const int u = (row & 63) >> 3;
+#pragma unroll
+        for (int i = 0; i < kXMax; ++i) {
+          const float px = ex2_approx(tx[i]);
+          lx[i] += px;
+          *reinterpret_cast<__nv_bfloat16 *>(pxb + i * 128 + ((u ^ (i & 7)) << 4)) = __float2bfloat16_rn(px);
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_px_full + 8 * (gx & 1));
+      }
+      if (!ok) break;
+      gx0 += n_tiles;
+      // ---- epilogue: column sums over all keys, then O_x^T / sum ----
+#pragma unroll
+      for (int i = 0; i < kXMax; ++i) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) lx[i] += __shfl_xor_sync(0xffffffffu, lx[i], o);
+      }
+      if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < kXMax; ++i) xcol_s[xw * kXMax + i] = lx[i];
+      }
+      ok = sync_y();
+      if (!ok) break;
+#pragma unroll
+      for (int i = 0; i < kXMax; ++i)
+        lx[i] = (xcol_s[0 * kXMax + i] + xcol_s[1 * kXMax + i]) + (xcol_s[2 * kXMax + i] + xcol_s[3 * kXMax + i]);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full, k & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
-      uint32_t s[128];
-      {
-        const uint32_t ta = lane_base + ((j & 1) ? G_::kTmemS1 : G_::kTmemS0);
-        tmem_ld32(ta, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-        tmem_ld32(ta + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-        tmem_ld32(ta + 64, *reinterpret_cast<uint32_t(*)[32]>(&s[64]));
-        tmem_ld32(ta + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
-        tmem_wait_ld();
-      }
+      uint32_t ox[kXMax];
+      tmem_ld8(lane_base + G_::kTmemOx, ox);
+      tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_s_free + 8 * (j & 1));
-      // columns past the end of a partial tile do not exist
-      const int valid = (j < n_pre) ? min(kBlockN, prm.P - j * kBlockN) : min(kBlockN, prm.Lq - (j - n_pre) * kBlockN);
-      if (valid < kBlockN) {
+      if (lane == 0) mbar_arrive(bar_ox_free);
+      // xcol_s is free again only when everyone has read it
+      ok = sync_y();
+      if (!ok) break;
+      __nv_bfloat16 *outp = reinterpret_cast<__nv_bfloat16 *>(prm.out) + it.b * prm.out_stride[0];
 #pragma unroll
-        for (int k = 0; k < 128; ++k)
-          if (k >= valid) s[k] = 0xff800000u;  // -inf
+      for (int i = 0; i < kXMax; ++i) {
+        if (i < it.x_rows) {
+          const int R = (it.mt + 1) * kBlockM + i;
+          const int hq = it.hk * prm.G + R / prm.Lq, ii = R % prm.Lq;
+          outp[hq * prm.out_stride[1] + (long long)ii * prm.out_stride[2] + row] =
+              __float2bfloat16_rn(__uint_as_float(ox[i]) / lx[i]);
+          if (prm.lse && row == 0)
+            prm.lse[((long long)it.b * prm.Hq + hq) * prm.Lq + ii] = (mref[i] + log2f(lx[i])) * kLn2;
+        }
       }
-      float mx = __uint_as_float(s[0]);
-#pragma unroll
-      for (int k = 1; k < 128; ++k) mx = fmaxf(mx, __uint_as_float(s[k]));
-      const float m_tile = mx * c2;
-      float factor = 1.f;
-      if (m_tile > m_used + kRescaleThreshold || m_used == -INFINITY) {
-        factor = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_tile);
-        m_used = m_tile;
-      }
-      const bool warp_rescales = __any_sync(0xffffffffu, factor != 1.f) && (j > 0);
-      l_sum *= factor;
-      float l0 = 0.f, l1 = 0.f;
-      const float neg_m = -m_used;
-      uint32_t pk[64];
-#pragma unroll
-      for (int k = 0; k < 64; ++k) {
-        const float p0 = ex2_approx(fmaf(__uint_as_float(s[2 * k]), c2, neg_m));
-        const float p1 = ex2_approx(fmaf(__uint_as_float(s[2 * k + 1]), c2, neg_m));
-        pk[k] = pack_bf16(p0, p1);
-        // normalise with the bf16 values the MMA will actually use: sum_j p~_j v_j / sum_j p~_j is then a
-        // convex combination of value rows whatever the rounding of p was
-        l0 += bf16lo_to_f32(pk[k]);
-        l1 += bf16hi_to_f32(pk[k]);
-      }
-      l_sum += l0 + l1;
-      if (j > 0) {
-        // P buffer free and O quiescent once the previous P V has completed
-        ok = mbar_wait(bar_pv_done, (j - 1) & 1, abort_flag);
+    }
+    timed_out = !ok;
+  } else {
+    // ============================ softmax + epilogue ============================
+    const int half = lane >> 4;                            // column half this thread works on
+    const int lane0 = (warp & 3) * 32 + (warp >> 2) * 16;   // first TMEM lane of this warp
+    const int row = lane0 + (lane & 15);                   // TMEM lane = row of the M-tile
+    const uint32_t lane_base = tmem + ((uint32_t)lane0 << 16);
+    const float c2 = prm.scale_log2;
+    constexpr int kOCols = D / 2;                          // accumulator columns per thread
+    const bool tracer = (warp & 3) == 0 && lane == 0;
+    (void)tracer;
+    bool ok = true;
+    int g0 = 0, k = 0;
+    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
+      const Item it = decode_item(prm, item);
+      const bool live = row < it.m_rows;
+      float m_used = -INFINITY;  // maximum the probabilities are expressed against (log2 units)
+      float l_sum = 0.f;         // this thread's half of the row sum
+      for (int j = 0; j < n_tiles; ++j) {
+        const int g = g0 + j;
+        ok = mbar_wait(bar_s_full + 8 * (g & 1), (g >> 1) & 1, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        if (warp_rescales) {
+        if (tracer) DS_TR(2 + (warp >> 2), g, 0);
+        const uint32_t s_base = lane_base + ((g & 1) ? G_::kTmemS1 : G_::kTmemS0);
+        uint32_t s[64];
+        tmem_ld16x2_32<64>(s_base, &s[0]);        // columns 64 half + 0..31
+        tmem_ld16x2_32<64>(s_base + 32, &s[32]);  // columns 64 half + 32..63
+        tmem_wait_ld();
+        if (tracer) DS_TR(2 + (warp >> 2), g, 1);
+        // columns past the end of a partial tile do not exist
+        const int valid = (j < n_pre) ? min(kBlockN, prm.P - j * kBlockN) : min(kBlockN, prm.Lq - (j - n_pre) * kBlockN);
+        if (valid < kBlockN) {
 #pragma unroll
-          for (int cb = 0; cb < D; cb += 32) {
+          for (int c = 0; c < 64; ++c)
+            if (c + 64 * half >= valid) s[c] = 0xff800000u;  // -inf
+        }
+        // row maximum: eight independent chains over this half, then the other half by shuffle
+        float mx;
+        {
+          float a[8];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) a[c] = __uint_as_float(s[c]);
+#pragma unroll
+          for (int c = 8; c < 56; c += 16) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              a[u] = fmax3(a[u], __uint_as_float(s[c + u]), __uint_as_float(s[c + 8 + u]));
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) a[u] = fmaxf(a[u], __uint_as_float(s[56 + u]));
+          mx = fmaxf(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]));
+          mx = fmax3(mx, a[6], a[7]);
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+        }
+        if (tracer) DS_TR(2 + (warp >> 2), g, 2);
+        const float m_tile = mx * c2;
+        float factor = 1.f;
+        if (m_tile > m_used + kRescaleThreshold || m_used == -INFINITY) {
+          factor = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_tile);
+          m_used = m_tile;
+        }
+        const bool warp_rescales = __any_sync(0xffffffffu, live && factor != 1.f) && (j > 0);
+        l_sum *= factor;
+        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+        const float neg_m = -m_used;
+        uint32_t pk[32];
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const float p0 = ex2_approx(fmaf(__uint_as_float(s[2 * c]), c2, neg_m));
+          const float p1 = ex2_approx(fmaf(__uint_as_float(s[2 * c + 1]), c2, neg_m));
+          const float p2 = ex2_approx(fmaf(__uint_as_float(s[2 * c + 2]), c2, neg_m));
+          const float p3 = ex2_approx(fmaf(__uint_as_float(s[2 * c + 3]), c2, neg_m));
+          pk[c] = pack_bf16(p0, p1);
+          pk[c + 1] = pack_bf16(p2, p3);
+          l0 += p0;
+          l1 += p1;
+          l2 += p2;
+          l3 += p3;
+        }
+        l_sum += (l0 + l1) + (l2 + l3);
+        if (tracer) DS_TR(2 + (warp >> 2), g, 3);
+        if (warp_rescales) {
+          // O must be quiescent: the previous P V has completed
+          ok = mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int cb = 0; cb < kOCols; cb += 32) {
             uint32_t o[32];
-            tmem_ld32(lane_base + G_::kTmemO + cb, o);
+            tmem_ld16x2_32<kOCols>(lane_base + G_::kTmemO + cb, o);
             tmem_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * factor);
-            tmem_st32(lane_base + G_::kTmemO + cb, o);
+            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor);
+            tmem_st16x2_32<kOCols>(lane_base + G_::kTmemO + cb, o);
           }
-          tmem_wait_st();
         }
+        if (tracer) DS_TR(2 + (warp >> 2), g, 4);
+        // P row -> TMEM over the first 64 columns of its own S buffer (two bf16 per column); this
+        // thread's 64 keys are columns 32 half .. 32 half + 31
+        tmem_st16x2_32<32>(s_base, pk);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_p_full + 8 * (g & 1));
+        if (tracer) DS_TR(2 + (warp >> 2), g, 5);
       }
-      // P row -> shared memory, K-major 128-byte swizzle: 16-byte unit u of a 128-byte row lands at u ^ (row % 8)
+      if (!ok) break;
+      // ---- epilogue of the item ----
+      l_sum += __shfl_xor_sync(0xffffffffu, l_sum, 16);
+      // the last P V of the item has completed (its own barrier, waited on once per item by everyone)
+      ok = mbar_wait(bar_o_full, k & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t o[kOCols];
 #pragma unroll
-      for (int g = 0; g < 16; ++g) {
-        const int c = g >> 3, u = g & 7;
-        *reinterpret_cast<uint4 *>(p_row + c * kChunkBytes + ((u ^ (row & 7)) << 4)) =
-            make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
-      }
-      fence_proxy_async();
+      for (int cb = 0; cb < kOCols; cb += 32) tmem_ld16x2_32<kOCols>(lane_base + G_::kTmemO + cb, &o[cb]);
+      tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_p_full);
-    }
-    if (ok) {
-      ok = mbar_wait(bar_pv_done, (n_tiles - 1) & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-    }
-    if (ok) {
-      tc_fence_after();
-      const int R = mt * kBlockM + row;
-      const bool live = row < m_rows;
-      const int hq = hk * prm.G + (live ? R / prm.Lq : 0), i = live ? R % prm.Lq : 0;
-      const float inv = 1.f / l_sum;
-      __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(prm.out) + b * prm.out_stride[0] + hq * prm.out_stride[1] +
-                            (long long)i * prm.out_stride[2];
+      if (lane == 0) mbar_arrive(bar_o_free);
+      if (live) {
+        const int R = it.mt * kBlockM + row;
+        const int hq = it.hk * prm.G + R / prm.Lq, i = R % prm.Lq;
+        const float inv = 1.f / l_sum;
+        __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(prm.out) + it.b * prm.out_stride[0] +
+                              hq * prm.out_stride[1] + (long long)i * prm.out_stride[2] + kOCols * half;
 #pragma unroll
-      for (int cb = 0; cb < D; cb += 32) {
-        uint32_t o[32];
-        tmem_ld32(lane_base + G_::kTmemO + cb, o);
-        tmem_wait_ld();
-        if (live) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 w;
-            w.x = pack_bf16(__uint_as_float(o[8 * g + 0]) * inv, __uint_as_float(o[8 * g + 1]) * inv);
-            w.y = pack_bf16(__uint_as_float(o[8 * g + 2]) * inv, __uint_as_float(o[8 * g + 3]) * inv);
-            w.z = pack_bf16(__uint_as_float(o[8 * g + 4]) * inv, __uint_as_float(o[8 * g + 5]) * inv);
-            w.w = pack_bf16(__uint_as_float(o[8 * g + 6]) * inv, __uint_as_float(o[8 * g + 7]) * inv);
-            *reinterpret_cast<uint4 *>(orow + cb + 8 * g) = w;
-          }
+        for (int c = 0; c < kOCols; c += 8) {
+          uint4 w;
+          w.x = pack_bf16(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+          w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+          w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+          w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+          *reinterpret_cast<uint4 *>(orow + c) = w;
         }
+        if (prm.lse && half == 0) prm.lse[((long long)it.b * prm.Hq + hq) * prm.Lq + i] = (m_used + log2f(l_sum)) * kLn2;
       }
-      if (live && prm.lse) prm.lse[((long long)b * prm.Hq + hq) * prm.Lq + i] = (m_used + log2f(l_sum)) * kLn2;
-      tc_fence_before();
     }
     timed_out = !ok;
   }
@@ -508,7 +1035,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
   if (timed_out && prm.status) atomicOr(prm.status, DS_DEV_TIMEOUT);
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
     tmem_dealloc(tmem, G_::kTmemCols);
   }
@@ -553,14 +1080,8 @@ bool make_map(CUtensorMap *m, const void *base, int D, long long rows, int H, in
 
 template <int D>
 int launch_d(const ds_attn_params &p, cudaStream_t stream) {
-  static std::once_flag once;
-  static cudaError_t attr_rc = cudaSuccess;
-  std::call_once(once, [] {
-    attr_rc = cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes);
-  });
-  // the attribute is per device: set it again when the current device changed (cheap)
+  // the attribute is per device: set it at every launch (cheap)
   DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes));
-  (void)attr_rc;
   TcParams prm;
   memset(&prm, 0, sizeof(prm));
   bool ok = true;
@@ -583,8 +1104,21 @@ int launch_d(const ds_attn_params &p, cudaStream_t stream) {
   prm.status = p.status;
   prm.B = p.B, prm.Hq = p.Hq, prm.Hkv = p.Hkv, prm.G = p.Hq / p.Hkv, prm.P = p.P, prm.T = p.T, prm.Lq = p.Lq;
   prm.scale_log2 = p.scale * kLog2e;
-  const int n_mtiles = ceil_div((long long)prm.G * p.Lq, kBlockM);
-  const dim3 grid(n_mtiles, p.Hkv, p.B);
+  // stacked query rows of one KV head: full 128-row tiles, and a remainder that either rides along
+  // with the last full tile (1..kXMax rows, D = 128) or gets a tile of its own
+  const long long rows_total = (long long)prm.G * p.Lq;
+  const int n_full = (int)(rows_total / kBlockM), rem = (int)(rows_total % kBlockM);
+  if (D == 128 && n_full >= 1 && rem >= 1 && rem <= kXMax) {
+    prm.n_mtiles = n_full;
+    prm.x_rows = rem;
+  } else {
+    prm.n_mtiles = n_full + (rem ? 1 : 0);
+    prm.x_rows = 0;
+  }
+  const long long n_items = (long long)p.B * p.Hkv * prm.n_mtiles;
+  if (n_items > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
+  prm.n_items = (int)n_items;
+  const int grid = (int)(n_items < sm_count() ? n_items : sm_count());
   attn_tc_kernel<D><<<grid, kNumThreads, Geo<D>::kSmemBytes, stream>>>(prm);
   DS_CUDA_OK(cudaGetLastError());
   note_launch(1);
@@ -593,10 +1127,15 @@ int launch_d(const ds_attn_params &p, cudaStream_t stream) {
 
 }  // namespace
 
+#ifdef DS_TRACE
+extern "C" __attribute__((visibility("default"))) int ds_debug_trace(long long *host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : 1;
+}
+#endif
+
 bool attn_tc_supported(const ds_attn_params &p) {
   if (p.dtype != DS_BF16 || (p.D != 64 && p.D != 128)) return false;
   if (!(p.scale > 0.f) || p.scale > 1e30f) return false;  // the running maximum assumes a positive scale
-  if (p.Hkv > 65535 || p.B > 65535) return false;
   if ((long long)(p.Hq / p.Hkv) * p.Lq > (1ll << 30)) return false;
   // TMA: 16-byte aligned bases and strides are already guaranteed by validation; extents must fit 32 bits
   return true;

@@ -42,10 +42,13 @@ def _compare(out, ref, dtype, what=""):
     return err, rms
 
 
-def _run_small(B, Hq, Hkv, D, P, T, idx, dtype, seed=0, q_scale=1.0, want_lse=True, noncontig=False):
+def _run_small(B, Hq, Hkv, D, P, T, idx, dtype, seed=0, q_scale=1.0, want_lse=True, noncontig=False,
+               k_boost=None):
     cfg = wl.StepConfig("t", B=B, Hq=Hq, Hkv=Hkv, D=D, P=P, gen=T, K=1, w=0, keep_last=False,
                         dtype="f32" if dtype == torch.float32 else "bf16", V=8, spike_p=0, seed=seed)
     x = wl.attention_inputs(cfg, device=DEV, q_scale=q_scale)
+    if k_boost is not None:      # (first prefix row, factor): later keys score far higher than earlier ones
+        x["k_pre"][:, :, k_boost[0]:] *= k_boost[1]
     if noncontig:   # strided views: padded rows and a head-major parent
         for k in list(x):
             t = x[k]
@@ -91,6 +94,37 @@ def test_gqa_head_grouping(D, G):
     T = 160
     idx = list(range(96)) + [T - 1]
     _run_small(2, 2 * G, 2, D, 300, T, idx, torch.bfloat16, seed=D + G)
+
+
+@pytest.mark.parametrize("G,Lq", [(1, 129), (1, 136), (1, 257), (2, 65), (4, 33), (7, 37), (3, 43)])
+def test_rows_beyond_the_last_full_tile(G, Lq):
+    """G * Lq = 128 m + r with r <= 8: the r rows are computed as a transposed side problem."""
+    T = 300
+    assert 1 <= (G * Lq) % 128 <= 8
+    idx = list(range(Lq - 1)) + [T - 1]
+    _run_small(2, 2 * G, 2, 128, 333, T, idx, torch.bfloat16, seed=G * 1000 + Lq)
+    _run_small(1, G, 1, 128, 0, T, idx, torch.bfloat16, seed=G * 1000 + Lq + 1)
+
+
+@pytest.mark.parametrize("boost_row", [128, 300, 640])
+def test_scores_that_grow_along_the_keys(boost_row):
+    """Later KV tiles score far above earlier ones: every running maximum and reference exponent has
+    to move (by much more than the lazy-rescale thresholds) after accumulation has started."""
+    T = 200
+    for Lq in (129, 64):
+        idx = list(range(Lq - 1)) + [T - 1]
+        _run_small(1, 2, 2, 128, 700, T, idx, torch.bfloat16, seed=boost_row + Lq, q_scale=3.0,
+                   k_boost=(boost_row, 5.0))
+
+
+def test_many_items_per_cta():
+    """More work items than SMs: every CTA runs several items back to back through one KV ring,
+    with and without the transposed side problem, and with both mixed (several M-tiles per head)."""
+    idx = list(range(128)) + [255]
+    _run_small(5, 64, 64, 128, 200, 256, idx, torch.bfloat16, seed=77, want_lse=True)
+    _run_small(3, 56, 8, 64, 130, 256, idx[:50], torch.bfloat16, seed=78)
+    _run_small(24, 12, 4, 128, 150, 256, idx[:43], torch.bfloat16, seed=79)     # 3 x 43 = 129 stacked rows
+    _run_small(40, 8, 4, 128, 300, 300, list(range(256)) + [299], torch.bfloat16, seed=80)  # 2 tiles + 2 extra rows
 
 
 def test_scattered_and_per_batch_index_lists():
