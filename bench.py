@@ -73,6 +73,31 @@ def conf_algorithmic_bytes(cfg):
 
 
 # --------------------------------------------------------------------------
+# replicas: the path has no exchange step, so N GPUs run N independent batches
+# --------------------------------------------------------------------------
+def rank_config(cfg, rank):
+    """The batch of one replica: same shapes, its own seeds."""
+    from paper_2601_17917_b200 import workloads as wl
+    return wl.shrink(cfg, seed=cfg.seed + 100000 * rank)
+
+
+def max_over_ranks(value, world, device):
+    """Slowest rank's time (the job's time).  The only collective of a multi-rank run, outside the timed region."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world, ms_per_step):
+    """Whole-job steps/s: every replica completes one step of its own batch per ms_per_step."""
+    return world * 1e3 / ms_per_step
+
+
+# --------------------------------------------------------------------------
 # clock sampling (read-only NVML)
 # --------------------------------------------------------------------------
 class ClockSampler:
@@ -421,7 +446,7 @@ def main():
 
     warmup = max(args.warmup, 3)
     # replicas: every rank draws its own batch (its rank offsets the seed); no data-path collective
-    rcfg = wl.shrink(cfg, seed=cfg.seed + 100000 * rank)
+    rcfg = rank_config(cfg, rank)
     step = Step(rcfg, device, stages=args.stages.split(","))
     sampler = ClockSampler(local)
     sampler.start()
@@ -431,12 +456,9 @@ def main():
     if extra:
         clocks["note"] = f"timed region + {extra} further identical steps"
     status = ds.ds_read_status(step.status)
-    if world > 1:
-        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, device)
     ms_per_step = total_ms / args.steps
-    value = world * 1e3 / ms_per_step
+    value = job_throughput(world, ms_per_step)
 
     e2e = None
     if not args.no_e2e and args.stages == "attn,confidence,select":
@@ -444,11 +466,8 @@ def main():
         del step.layers[1:]
         torch.cuda.empty_cache()
         e_ms, h2d, d2h = time_e2e(rcfg, device, e2e_steps, 3)
-        if world > 1:
-            t = torch.tensor([e_ms], device=device, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        e2e = {"value": world * 1e3 / e_ms, "unit": "steps/s", "h2d_bytes_per_step": int(h2d),
+        e_ms = max_over_ranks(e_ms, world, device)
+        e2e = {"value": job_throughput(world, e_ms), "unit": "steps/s", "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "ms_per_step": e_ms, "steps": e2e_steps,
                "layout": "tail rows shipped compact (T = Lq): only what the step reads crosses the link"}
 
