@@ -27,9 +27,11 @@
 //              without extra rows), kept apart so that its cross-warp agreement never sits on the
 //              main rows' critical path
 //   warp 14    issues P V.  Issuing blocks while the tensor pipe's queue is full, so the two streams
-//              have an issuer each and Q K^T runs as far ahead as the double-buffered S allows.
+//              have an issuer each; the one dependency the pipe no longer orders by itself (Q K^T of
+//              tile g + 2 overwrites the buffer P V of tile g reads) is an explicit barrier wait.
 // Per KV tile:  S[g%2] = Q K^T            (tcgen05.mma, both operands K-major in shared memory)
-//               softmax warps: tcgen05.ld S, row maximum, P = 2^(s*c - m) as bf16 written to TMEM
+//               softmax warps: tcgen05.ld S, row maximum, P = 2^(s*c - m) as bf16 written over the
+//               first 64 columns of the same S buffer
 //               O += P V                   (A = P from TMEM, B = V MN-major straight from its [kv][D]
 //                                           layout)
 // S/P is double buffered so Q K^T of the next tile runs under the softmax of this one.  O is only
@@ -95,8 +97,8 @@ struct Geo {
   static constexpr int kOffRing = kOffPx + 4 * kXChunkBytes;
   static constexpr int kOffBar = kOffRing + kSlots * kTileBytes;
   // barriers: q_full, q_free, s_full[2], p_full[2], pv_done[2], o_free, xbar[2], ybar, o_full, px_full[2],
-  //           ox_free, sx_full[2], pvx_done[2], s_free[2], slot_full[kSlots], slot_empty[kSlots]
-  static constexpr int kNumBars = 22 + 2 * kSlots;
+  //           ox_free, sx_full[2], pvx_done[2], slot_full[kSlots], slot_empty[kSlots]
+  static constexpr int kNumBars = 20 + 2 * kSlots;
   static constexpr int kOffIdx = kOffBar + 8 * kNumBars;     // int32[128] gathered-row indices of a KV tile
   static constexpr int kOffIdxQ = kOffIdx + 4 * 128;         // int32[128] gathered-row indices of a query tile
   static constexpr int kOffXflag = kOffIdxQ + 4 * 128;       // int[2 parity][4 warps]
@@ -105,16 +107,14 @@ struct Geo {
   static constexpr int kOffMisc = kOffIdxCache + 4 * kIdxCap;  // tmem base, abort flag
   static constexpr int kSmemBytes = kOffMisc + 16 + 1024;    // + slack to align the base to 1024
   static constexpr int kTmemCols = 512;
-  static constexpr int kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256, kTmemP = 384;  // P: 128 bf16 = 64 columns
-  static constexpr int kTmemSx0 = 448, kTmemSx1 = 464, kTmemOx = 480;
+  static constexpr int kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;  // P(g) overwrites columns 0..63 of S(g)
+  static constexpr int kTmemSx0 = 384, kTmemSx1 = 400, kTmemOx = 416;
 };
 static_assert(Geo<128>::kSmemBytes <= 227 * 1024, "shared memory budget");
 static_assert(Geo<64>::kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct TcParams {
-  // 5-D views {64 columns, rows, 64-column chunk, head, batch}; the number is the box height in rows.
-  // A 128-row box spans all chunks (one copy fills a whole tile); smaller boxes take one chunk.
-  CUtensorMap kpre, vpre, k128, k32, k1, v128, v32, v1, q128, q32, q1;
+  CUtensorMap kpre, vpre, k32, k1, v32, v1, q32, q1;
   const int32_t *idx;
   long long idx_bstride;
   void *out;
@@ -198,11 +198,11 @@ __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarr
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3, int c4) {
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
   asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
       : "memory");
 }
 
@@ -304,14 +304,11 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) { return fmaxf
 // period is Lq) into a swizzled tile whose 64-column chunks are chunk_stride bytes apart.  The whole
 // warp calls it; lane 0 issues the copies.  Returns the bytes issued (valid on lane 0).
 // ------------------------------------------------------------------------------------------------
-struct RowMaps {
-  const CUtensorMap *m128, *m32, *m1;
-};
 template <int D>
-__device__ __forceinline__ uint32_t gather_rows(const TcParams &prm, const RowMaps maps, uint32_t dst,
-                                                uint32_t chunk_stride, uint32_t bar, int R0, int n, int head0, int b,
-                                                int32_t *idx_s, const int32_t *idx_cache, bool &bad_index,
-                                                bool staged = false) {
+__device__ __forceinline__ uint32_t gather_rows(const TcParams &prm, const CUtensorMap *map32, const CUtensorMap *map1,
+                                                uint32_t dst, uint32_t chunk_stride, uint32_t bar, int R0, int n,
+                                                int head0, int b, int32_t *idx_s, const int32_t *idx_cache,
+                                                bool &bad_index, bool staged = false) {
   const int lane = threadIdx.x & 31;
   const int Lq = prm.Lq;
   // position of logical row R0 inside its head; divisions only when the stacking actually wraps
@@ -345,25 +342,15 @@ __device__ __forceinline__ uint32_t gather_rows(const TcParams &prm, const RowMa
     int r = 0, pos = pos0;
     while (r < n) {
       const int row = idx_s[r];
-      // the longest run of consecutive rows a box covers: a whole tile, 32 rows, or one
-      int step = 1;
-      if ((r & 7) == 0) {
-        if (r == 0 && n == kBlockN && chunk_stride == kChunkBytes && pos + kBlockN <= Lq && idx_s[kBlockN - 1] - row == kBlockN - 1)
-          step = kBlockN;
-        else if (r + 32 <= n && pos + 32 <= Lq && idx_s[r + 31] - row == 31)
-          step = 32;
-      }
-      if (step == kBlockN) {
-        tma_load_5d(dst, maps.m128, bar, 0, row, 0, head, b);
-      } else {
+      const bool box32 = ((r & 7) == 0) && (r + 32 <= n) && (pos + 32 <= Lq) && (idx_s[r + 31] - row == 31);
+      const int step = box32 ? 32 : 1;
 #pragma unroll
-        for (int c = 0; c < Geo<D>::kChunks; ++c)
-          tma_load_5d(dst + c * chunk_stride + r * 128, step == 32 ? maps.m32 : maps.m1, bar, 0, row, c, head, b);
-      }
+      for (int c = 0; c < Geo<D>::kChunks; ++c)
+        tma_load_4d(dst + c * chunk_stride + r * 128, box32 ? map32 : map1, bar, c * 64, row, head, b);
       bytes += (uint32_t)step * 128u * Geo<D>::kChunks;
       r += step;
       pos += step;
-      if (pos >= Lq) {  // a box never crosses a head, so this is at most one wrap
+      if (pos >= Lq) {  // a 32-row box never crosses a head, so this is at most one wrap
         pos -= Lq;
         ++head;
       }
@@ -412,8 +399,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
   const uint32_t bar_ox_free = bar0 + 120;   // the epilogue has read O_x^T
   const uint32_t bar_sx_full = bar0 + 128;   // [2] S_x^T of a tile is in TMEM
   const uint32_t bar_pvx_done = bar0 + 144;  // [2] O_x^T += V^T P_x^T of a tile has completed
-  const uint32_t bar_s_free = bar0 + 160;    // [2] the softmax warps hold S of a tile in registers
-  const uint32_t bar_slot_full = bar0 + 176;                       // [kSlots]
+  const uint32_t bar_slot_full = bar0 + 160;                       // [kSlots]
   const uint32_t bar_slot_empty = bar_slot_full + 8 * G_::kSlots;  // [kSlots]
   int32_t *idx_s = reinterpret_cast<int32_t *>(smem + G_::kOffIdx);
   int32_t *idxq_s = reinterpret_cast<int32_t *>(smem + G_::kOffIdxQ);
@@ -445,8 +431,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     mbar_init(bar_sx_full + 8, 1);
     mbar_init(bar_pvx_done, 1);
     mbar_init(bar_pvx_done + 8, 1);
-    mbar_init(bar_s_free, kSoftmaxWarps);
-    mbar_init(bar_s_free + 8, kSoftmaxWarps);
     for (int s = 0; s < G_::kSlots; ++s) {
       mbar_init(bar_slot_full + 8 * s, 1);
       mbar_init(bar_slot_empty + 8 * s, 1);
@@ -472,13 +456,10 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         prefetch_map(&prm.kpre);
         prefetch_map(&prm.vpre);
       }
-      prefetch_map(&prm.k128);
       prefetch_map(&prm.k32);
       prefetch_map(&prm.k1);
-      prefetch_map(&prm.v128);
       prefetch_map(&prm.v32);
       prefetch_map(&prm.v1);
-      prefetch_map(&prm.q128);
       prefetch_map(&prm.q32);
       prefetch_map(&prm.q1);
     }
@@ -497,23 +478,20 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       __syncwarp();
       idx_cache = cache;
     }
-    const RowMaps q_maps = {&prm.q128, &prm.q32, &prm.q1};
-    const RowMaps k_maps = {&prm.k128, &prm.k32, &prm.k1};
-    const RowMaps v_maps = {&prm.v128, &prm.v32, &prm.v1};
     const int n_my = (prm.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // items of this CTA
     int q_next = 0;  // first item (in this CTA's order) whose query tile has not been requested yet
     // Requests the query tile(s) of this CTA's kq-th item.  The caller has made sure the previous
     // item's last Q K^T has completed.
     auto issue_q = [&](int kq) {
       const Item it = decode_item(prm, blockIdx.x + kq * gridDim.x);
-      uint32_t bytes = gather_rows<D>(prm, q_maps, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
+      uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
                                       it.mt * kBlockM, it.m_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
       if (it.x_rows > 0) {
         // rows of the small query tile that are not loaded must be finite: clear the tile first
         for (int q = lane; q < (2 * kXChunkBytes) / 16; q += 32)
           *reinterpret_cast<uint4 *>(smem + G_::kOffQx + q * 16) = make_uint4(0, 0, 0, 0);
         fence_proxy_async();
-        bytes += gather_rows<D>(prm, q_maps, sbase + G_::kOffQx, kXChunkBytes, bar_q_full,
+        bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, sbase + G_::kOffQx, kXChunkBytes, bar_q_full,
                                 (it.mt + 1) * kBlockM, it.x_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
       }
       if (lane == 0) mbar_arrive_expect_tx(bar_q_full, bytes);
@@ -560,17 +538,20 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           DS_TR(0, issued >> 1, kv * 3 + 1);
           if (j < n_pre) {
             if (lane == 0) {
-              tma_load_5d(dst, kv ? &prm.vpre : &prm.kpre, full, 0, j * kBlockN, 0, it.hk, it.b);
+              const CUtensorMap *map = kv ? &prm.vpre : &prm.kpre;
+#pragma unroll
+              for (int c = 0; c < G_::kChunks; ++c)
+                tma_load_4d(dst + c * kChunkBytes, map, full, c * 64, j * kBlockN, it.hk, it.b);
               mbar_arrive_expect_tx(full, G_::kTileBytes);
             }
           } else {
             const int t0 = (j - n_pre) * kBlockN;
             const int n = min(kBlockN, prm.Lq - t0);
-            if (kv == 1 && (n & 15) != 0) {
-              // P V runs over whole 16-key steps: the rows that fill up the last step meet P = 0 in the
-              // MMA and must be zero, not stale (a row of a chunk is 8 x 16 bytes: 4 rows per pass)
+            if (kv == 1 && n < kBlockN) {
+              // rows past the end of a V tile meet P = 0 in the MMA: make them zero, not stale
+              // (a row of a chunk is 8 x 16 bytes: 4 rows per pass of the warp)
               uint8_t *tile = smem + G_::kOffRing + slot * G_::kTileBytes + (lane & 7) * 16;
-              for (int row = n + (lane >> 3); row < ((n + 15) & ~15); row += 4) {
+              for (int row = n + (lane >> 3); row < kBlockN; row += 4) {
 #pragma unroll
                 for (int c = 0; c < G_::kChunks; ++c)
                   *reinterpret_cast<uint4 *>(tile + c * kChunkBytes + row * 128) = make_uint4(0, 0, 0, 0);
@@ -578,8 +559,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
               fence_proxy_async();
             }
             // the V fill of a tile directly follows its K fill: the staged row list is still valid
-            const uint32_t bytes = gather_rows<D>(prm, kv ? v_maps : k_maps, dst, kChunkBytes, full, t0, n, it.hk, it.b,
-                                                  idx_s, idx_cache, bad_index, kv == 1);
+            const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, dst, kChunkBytes,
+                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, bad_index, kv == 1);
             if (lane == 0) mbar_arrive_expect_tx(full, bytes);
           }
           DS_TR(0, issued >> 1, kv * 3 + 2);
@@ -626,10 +607,11 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int g = g0 + j, gx = gx0 + j;
         const int fill = 2 * g, slot = fill % G_::kSlots, use = fill / G_::kSlots;
-        // the K tile has landed, and S[g % 2] is free: the softmax warps have loaded tile g - 2 from it
+        // the K tile has landed, and S[g % 2] is free: P V of tile g - 2, the reader of the P it still
+        // holds, has completed
         bool w;
         if (g >= 2)
-          w = mbar_wait2(bar_slot_full + 8 * slot, use & 1, bar_s_free + 8 * (g & 1), ((g - 2) >> 1) & 1, abort_flag);
+          w = mbar_wait2(bar_slot_full + 8 * slot, use & 1, bar_pv_done + 8 * (g & 1), ((g - 2) >> 1) & 1, abort_flag);
         else
           w = mbar_wait(bar_slot_full + 8 * slot, use & 1, abort_flag);
         if (!__all_sync(0xffffffffu, w)) {
@@ -703,18 +685,13 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         }
         tc_fence_after();
         const uint64_t dv = dv0 + (uint64_t)((slot * G_::kTileBytes) >> 4);
-        // 16-key steps of this tile that hold keys (a partial tile ends early; the rows that fill up its
-        // last step are zero)
-        const int valid = (j < n_pre) ? min(kBlockN, prm.P - j * kBlockN) : min(kBlockN, prm.Lq - (j - n_pre) * kBlockN);
-        const int n_ks = (valid + 15) >> 4;
         if (elect_one()) {
           DS_TR(1, g, 2);
 #pragma unroll
           for (int ks = 0; ks < kBlockN / 16; ++ks)
-            if (ks < n_ks)
-              umma_ts(tm + G_::kTmemO, tm + G_::kTmemP + ks * 8, dv + ((ks * 2048) >> 4), idesc_pv,
-                      (j > 0 || ks > 0) ? 1u : 0u);
-          umma_commit(bar_pv_done + 8 * (g & 1));  // P may be overwritten, O may be rescaled
+            umma_ts(tm + G_::kTmemO, tm + ((g & 1) ? G_::kTmemS1 : G_::kTmemS0) + ks * 8, dv + ((ks * 2048) >> 4),
+                    idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+          umma_commit(bar_pv_done + 8 * (g & 1));  // frees S[g % 2] for Q K^T of tile g + 2
         }
         __syncwarp();
         if (has_x) {
@@ -733,8 +710,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
 #pragma unroll
               for (int ks = 0; ks < kBlockN / 16; ++ks) {
                 const uint32_t offx = ((gx & 1) * 2 * kXChunkBytes + (ks / 4) * kXChunkBytes + (ks % 4) * 32) >> 4;
-                if (ks < n_ks)
-                  umma_ss(tm + G_::kTmemOx, dv + ((ks * 2048) >> 4), dpx + offx, idesc_pv_x, (j > 0 || ks > 0) ? 1u : 0u);
+                umma_ss(tm + G_::kTmemOx, dv + ((ks * 2048) >> 4), dpx + offx, idesc_pv_x, (j > 0 || ks > 0) ? 1u : 0u);
               }
               umma_commit(bar_pvx_done + 8 * (gx & 1));
             }
@@ -941,9 +917,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         tmem_ld16x2_32<64>(s_base, &s[0]);        // columns 64 half + 0..31
         tmem_ld16x2_32<64>(s_base + 32, &s[32]);  // columns 64 half + 32..63
         tmem_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_s_free + 8 * (g & 1));
         if (tracer) DS_TR(2 + (warp >> 2), g, 1);
         // columns past the end of a partial tile do not exist
         const int valid = (j < n_pre) ? min(kBlockN, prm.P - j * kBlockN) : min(kBlockN, prm.Lq - (j - n_pre) * kBlockN);
@@ -997,28 +970,26 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         }
         l_sum += (l0 + l1) + (l2 + l3);
         if (tracer) DS_TR(2 + (warp >> 2), g, 3);
-        if (j > 0) {
-          // P is free and O quiescent once the previous P V has completed (at the first tile of an item
-          // the epilogue of the previous item has already seen that)
+        if (warp_rescales) {
+          // O must be quiescent: the previous P V has completed
           ok = mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
-          if (warp_rescales) {
 #pragma unroll
-            for (int cb = 0; cb < kOCols; cb += 32) {
-              uint32_t o[32];
-              tmem_ld16x2_32<kOCols>(lane_base + G_::kTmemO + cb, o);
-              tmem_wait_ld();
+          for (int cb = 0; cb < kOCols; cb += 32) {
+            uint32_t o[32];
+            tmem_ld16x2_32<kOCols>(lane_base + G_::kTmemO + cb, o);
+            tmem_wait_ld();
 #pragma unroll
-              for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor);
-              tmem_st16x2_32<kOCols>(lane_base + G_::kTmemO + cb, o);
-            }
+            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor);
+            tmem_st16x2_32<kOCols>(lane_base + G_::kTmemO + cb, o);
           }
         }
         if (tracer) DS_TR(2 + (warp >> 2), g, 4);
-        // P row -> TMEM, two bf16 per column; this thread's 64 keys are columns 32 half .. 32 half + 31
-        tmem_st16x2_32<32>(lane_base + G_::kTmemP, pk);
+        // P row -> TMEM over the first 64 columns of its own S buffer (two bf16 per column); this
+        // thread's 64 keys are columns 32 half .. 32 half + 31
+        tmem_st16x2_32<32>(s_base, pk);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -1092,19 +1063,17 @@ EncodeFn encode_fn() {
   return fn;
 }
 
-// [B][H][rows][D] bf16 tensor with element strides {batch, head, row}, seen as
-// {64 columns, rows, D/64 chunks, H, B}; box = 64 columns x box_rows rows x box_chunks chunks.
-bool make_map(CUtensorMap *m, const void *base, int D, long long rows, int H, int B, const int64_t stride[3], int box_rows,
-              int box_chunks) {
+// [B][H][rows][D] bf16 tensor with element strides {batch, head, row}; box = 64 columns x box_rows rows.
+bool make_map(CUtensorMap *m, const void *base, int D, long long rows, int H, int B, const int64_t stride[3], int box_rows) {
   EncodeFn fn = encode_fn();
   if (!fn) return false;
-  const cuuint64_t dims[5] = {64, (cuuint64_t)rows, (cuuint64_t)(D / 64), (cuuint64_t)H, (cuuint64_t)B};
+  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)H, (cuuint64_t)B};
   // a dimension of extent 1 may carry any stride; keep them valid multiples of 16 bytes
-  const cuuint64_t strides[4] = {(cuuint64_t)stride[2] * 2, 128, (cuuint64_t)(H > 1 ? stride[1] : stride[2] * rows) * 2,
+  const cuuint64_t strides[3] = {(cuuint64_t)stride[2] * 2, (cuuint64_t)(H > 1 ? stride[1] : stride[2] * rows) * 2,
                                  (cuuint64_t)(B > 1 ? stride[0] : (H > 1 ? stride[1] * H : stride[2] * rows)) * 2};
-  const cuuint32_t box[5] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_chunks, 1, 1};
-  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), dims, strides, box, estr,
+  const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -1116,20 +1085,16 @@ int launch_d(const ds_attn_params &p, cudaStream_t stream) {
   TcParams prm;
   memset(&prm, 0, sizeof(prm));
   bool ok = true;
-  constexpr int kCh = D / 64;
   if (p.P > 0) {
-    ok = ok && make_map(&prm.kpre, p.k_prefix, D, p.P, p.Hkv, p.B, p.kv_prefix_stride, kBlockN, kCh);
-    ok = ok && make_map(&prm.vpre, p.v_prefix, D, p.P, p.Hkv, p.B, p.kv_prefix_stride, kBlockN, kCh);
+    ok = ok && make_map(&prm.kpre, p.k_prefix, D, p.P, p.Hkv, p.B, p.kv_prefix_stride, kBlockN);
+    ok = ok && make_map(&prm.vpre, p.v_prefix, D, p.P, p.Hkv, p.B, p.kv_prefix_stride, kBlockN);
   }
-  ok = ok && make_map(&prm.k128, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, kBlockN, kCh);
-  ok = ok && make_map(&prm.k32, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 32, 1);
-  ok = ok && make_map(&prm.k1, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 1, 1);
-  ok = ok && make_map(&prm.v128, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, kBlockN, kCh);
-  ok = ok && make_map(&prm.v32, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 32, 1);
-  ok = ok && make_map(&prm.v1, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 1, 1);
-  ok = ok && make_map(&prm.q128, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, kBlockN, kCh);
-  ok = ok && make_map(&prm.q32, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 32, 1);
-  ok = ok && make_map(&prm.q1, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 1, 1);
+  ok = ok && make_map(&prm.k32, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 32);
+  ok = ok && make_map(&prm.k1, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 1);
+  ok = ok && make_map(&prm.v32, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 32);
+  ok = ok && make_map(&prm.v1, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 1);
+  ok = ok && make_map(&prm.q32, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 32);
+  ok = ok && make_map(&prm.q1, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 1);
   if (!ok) return DS_ERR_CUDA;
   prm.idx = p.idx;
   prm.idx_bstride = p.idx_batch_stride;
