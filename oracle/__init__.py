@@ -14,6 +14,9 @@ Contents
   tail over prefix + whole tail, materialising every score row.  It exists to
   pin ``attn``: retaining every suffix position must reproduce it.
 * ``confidence`` (C, ``oracle_confidence``): Eq. 4.
+* ``lmhead_confidence`` (C, ``oracle_lmhead_confidence``): the output projection
+  (last of the "remaining model components" that turn attention outputs into
+  logits) composed with Eq. 4, logits kept in float64.
 * ``threshold`` / ``select`` (C, float32, contraction off): Eq. 10, Eq. 9, Eq. 5,
   block termination and the early-exit flag.
 
@@ -61,6 +64,9 @@ def _load():
             c_ip, ctypes.c_long, ctypes.c_double, c_dp, c_dp]
         lib.oracle_confidence.restype = ctypes.c_int
         lib.oracle_confidence.argtypes = [c_fp, ctypes.c_long, ctypes.c_long, ctypes.c_long, c_dp, c_ip]
+        lib.oracle_lmhead_confidence.restype = ctypes.c_int
+        lib.oracle_lmhead_confidence.argtypes = [c_fp, c_fp, ctypes.c_long, ctypes.c_long, ctypes.c_long, c_dp,
+                                                 c_ip, c_dp]
         lib.oracle_threshold.restype = ctypes.c_float
         lib.oracle_threshold.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_float,
                                          ctypes.c_float]
@@ -184,6 +190,26 @@ def confidence(logits):
     if rc != 0:
         raise ValueError("oracle_confidence rejected its arguments")
     return conf, tok
+
+
+def lmhead_confidence(hidden, weight, want_logits=False):
+    """Output projection z = hidden @ weight.T in float64 followed by Eq. 4, the logits never rounded or
+    stored in a narrower type.  hidden [rows, hid], weight [V, hid] (float32 values; bf16 widened exactly
+    by the caller).  Returns (conf float64 [rows], tok int32 [rows]) and, on request, the logits."""
+    lib = _load()
+    h, w = _f32(hidden), _f32(weight)
+    rows, hid = h.shape
+    V = w.shape[0]
+    assert w.shape == (V, hid)
+    conf = np.empty(rows, dtype=np.float64)
+    tok = np.empty(rows, dtype=np.int32)
+    z = np.empty((rows, V), dtype=np.float64) if want_logits else None
+    rc = lib.oracle_lmhead_confidence(_ptr(h, ctypes.c_float), _ptr(w, ctypes.c_float), rows, hid, V,
+                                      _ptr(conf, ctypes.c_double), _ptr(tok, ctypes.c_int32),
+                                      _ptr(z, ctypes.c_double) if want_logits else None)
+    if rc != 0:
+        raise ValueError("oracle_lmhead_confidence rejected its arguments")
+    return (conf, tok, z) if want_logits else (conf, tok)
 
 
 # --------------------------------------------------------------------------

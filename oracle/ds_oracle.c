@@ -229,3 +229,55 @@ int oracle_select(int B, int K, const float *conf, const int32_t *tok,
   *active_cnt = n_active;
   return 0;
 }
+
+/*
+ * Output projection followed by Eq. 4, without storing the logits.
+ *
+ * In the prediction forward the attention output is "processed by the
+ * remaining model components to produce the prediction logits" (Method,
+ * "Dynamic Confidence Aware Parallel Decoding"); the last of those components
+ * is the output projection z_r = W h_r.  Eq. 4 then reads c_r = max_j
+ * softmax(z_r)_j and x^_r = argmax_j z_rj.  This function is that composition
+ * written out: a plain matrix-vector product in double per row, then the same
+ * max / lowest-index argmax / sum of exponentials as oracle_confidence.
+ *
+ *   hidden  [rows][hid]  float32 (bf16 values widened exactly by the caller)
+ *   weight  [V][hid]     float32, row j is the output embedding of token j
+ *   conf    [rows]       double
+ *   tok     [rows]
+ *   logits  [rows][V]    double, may be NULL
+ */
+int oracle_lmhead_confidence(const float *hidden, const float *weight, long rows,
+                             long hid, long V, double *conf, int32_t *tok,
+                             double *logits) {
+  if (rows < 0 || hid <= 0 || V <= 0) return -1;
+  int bad = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long r = 0; r < rows; ++r) {
+    const float *h = hidden + r * hid;
+    double *z = logits ? logits + r * V : (double *)malloc(sizeof(double) * V);
+    if (!z) {
+      bad = 1;
+      continue;
+    }
+    for (long j = 0; j < V; ++j) {
+      const float *w = weight + j * hid;
+      double acc = 0.0;
+      for (long k = 0; k < hid; ++k) acc += (double)h[k] * (double)w[k];
+      z[j] = acc;
+    }
+    double m = z[0];
+    long arg = 0;
+    for (long j = 1; j < V; ++j)
+      if (z[j] > m) {
+        m = z[j];
+        arg = j;
+      }
+    double sum = 0.0;
+    for (long j = 0; j < V; ++j) sum += exp(z[j] - m);
+    conf[r] = 1.0 / sum;
+    tok[r] = (int32_t)arg;
+    if (!logits) free(z);
+  }
+  return bad ? -2 : 0;
+}
