@@ -144,6 +144,32 @@ DS_API int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_
                   void *workspace, size_t workspace_bytes, void *stream);
 
 /* ------------------------------------------------------------------------
+ * ds_lmhead_confidence  (output projection + Eq. 4, fused)
+ *
+ * In the prediction forward the attention outputs are "processed by the
+ * remaining model components to produce the prediction logits" (Method,
+ * "Dynamic Confidence Aware Parallel Decoding"); the last of them is the output
+ * projection z_r = W h_r.  This entry point computes, for every row r,
+ *     z_rj    = sum_k hidden[r][k] * weight[j][k]          (j < V, fp32 accumulation)
+ *     tok[r]  = lowest j with z_rj == max_j z_rj
+ *     conf[r] = 1 / sum_j exp(z_rj - max_j z_rj)            (Eq. 4)
+ * without ever writing the [rows x V] logits: they stay on chip as fp32
+ * accumulators (so, unlike ds_confidence on stored bf16 logits, they are not
+ * rounded to bf16 either).
+ *
+ * hidden [rows][ld_h] and weight [V][ld_w] are bf16, row-major, hid elements
+ * used per row; bases 16-byte aligned, ld_h, ld_w and hid multiples of 8.
+ * Workspace: ds_lmhead_confidence_workspace(rows, V) bytes, 256-byte aligned
+ * (one 16-byte partial result per row and per 256-token tile of the vocabulary).
+ * `status` (optional device word) receives DS_DEV_TIMEOUT if a bounded on-chip
+ * wait expires.  Errors: DS_ERR_INVALID_ARG, DS_ERR_WORKSPACE, DS_ERR_CUDA.
+ * ------------------------------------------------------------------------ */
+DS_API size_t ds_lmhead_confidence_workspace(int64_t rows, int64_t V);
+DS_API int ds_lmhead_confidence(const void *hidden, const void *weight, int64_t rows, int64_t hid, int64_t V,
+                         int64_t ld_h, int64_t ld_w, float *conf, int32_t *tok, void *workspace,
+                         size_t workspace_bytes, uint32_t *status, void *stream);
+
+/* ------------------------------------------------------------------------
  * ds_confidence_static  (no counterpart in the paper: a packaging variant)
  *
  * The same computation and the same kernel as ds_confidence, for callers that

@@ -18,7 +18,8 @@ from . import workloads  # noqa: F401  (seeded synthetic inputs)
 
 __all__ = [
     "lib", "retained_indices", "ds_attn_pruned", "ds_attn_pruned_workspace", "ds_confidence",
-    "ds_confidence_workspace", "ds_confidence_static", "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
+    "ds_confidence_workspace", "ds_confidence_static", "ds_lmhead_confidence", "ds_lmhead_confidence_workspace",
+    "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
     "ds_launch_count", "DsError", "DS_F32", "DS_BF16", "DS_DEV_INDEX", "DS_DEV_TIMEOUT",
 ]
 
@@ -81,6 +82,11 @@ def lib() -> ctypes.CDLL:
         L.ds_confidence.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.ds_lmhead_confidence_workspace.restype = ctypes.c_size_t
+        L.ds_lmhead_confidence_workspace.argtypes = [ctypes.c_int64, ctypes.c_int64]
+        L.ds_lmhead_confidence.restype = ctypes.c_int
+        L.ds_lmhead_confidence.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int64] * 5 + [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p]
         L.ds_confidence_static.restype = ctypes.c_int
         L.ds_confidence_static.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                            ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
@@ -235,6 +241,37 @@ def ds_confidence(logits, row_list=None, conf=None, tok=None, workspace=None, st
                              _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
     if rc != DS_OK:
         raise DsError(rc, "ds_confidence")
+    return conf, tok
+
+
+def ds_lmhead_confidence_workspace(rows: int, V: int) -> int:
+    return int(lib().ds_lmhead_confidence_workspace(int(rows), int(V)))
+
+
+def ds_lmhead_confidence(hidden, weight, conf=None, tok=None, workspace=None, status=None, stream=None):
+    """Output projection fused with Eq. 4: hidden bf16 [rows, hid], weight bf16 [V, hid] (last dimension
+    contiguous).  Returns (conf f32 [rows], tok i32 [rows]); the logits are never stored."""
+    _check_dev(hidden, weight, conf, tok, workspace, status)
+    if hidden.dtype != torch.bfloat16 or weight.dtype != torch.bfloat16:
+        raise TypeError("hidden and weight must be bf16")
+    if hidden.dim() != 2 or weight.dim() != 2 or hidden.stride(1) != 1 or weight.stride(1) != 1:
+        raise ValueError("hidden [rows, hid] and weight [V, hid] must have contiguous rows")
+    rows, hid = hidden.shape
+    V = weight.shape[0]
+    if weight.shape[1] != hid:
+        raise ValueError("hidden and weight disagree on the hidden size")
+    if conf is None:
+        conf = torch.empty(rows, dtype=torch.float32, device=hidden.device)
+    if tok is None:
+        tok = torch.empty(rows, dtype=torch.int32, device=hidden.device)
+    if workspace is None:
+        workspace = torch.empty(max(ds_lmhead_confidence_workspace(rows, V), 256), dtype=torch.uint8,
+                                device=hidden.device)
+    rc = lib().ds_lmhead_confidence(_ptr(hidden), _ptr(weight), rows, hid, V, hidden.stride(0), weight.stride(0),
+                                    _ptr(conf), _ptr(tok), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                    _ptr(status), _stream(stream))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_lmhead_confidence")
     return conf, tok
 
 

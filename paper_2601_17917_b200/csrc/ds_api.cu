@@ -114,6 +114,25 @@ int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_t V, in
                                workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
+size_t ds_lmhead_confidence_workspace(int64_t rows, int64_t V) { return ds::lmhead_workspace_bytes(rows, V); }
+
+int ds_lmhead_confidence(const void *hidden, const void *weight, int64_t rows, int64_t hid, int64_t V, int64_t ld_h,
+                         int64_t ld_w, float *conf, int32_t *tok, void *workspace, size_t workspace_bytes,
+                         uint32_t *status, void *stream) {
+  if (rows < 0 || hid <= 0 || V <= 0 || ld_h < hid || ld_w < hid) return DS_ERR_INVALID_ARG;
+  if (rows > 0x7fffffffLL || V > 0x7fffffffLL || hid > 0x7fffffffLL) return DS_ERR_INVALID_ARG;
+  if (rows == 0) return DS_OK;
+  if (!hidden || !weight || !conf || !tok) return DS_ERR_INVALID_ARG;
+  if (!ds::aligned(hidden, 16) || !ds::aligned(weight, 16) || !ds::aligned(conf, 4) || !ds::aligned(tok, 4) ||
+      (status && !ds::aligned(status, 4)))
+    return DS_ERR_INVALID_ARG;
+  if (hid % 8 != 0 || ld_h % 8 != 0 || ld_w % 8 != 0) return DS_ERR_INVALID_ARG;
+  const size_t need = ds::lmhead_workspace_bytes(rows, V);
+  if (!workspace || !ds::aligned(workspace, 256) || workspace_bytes < need) return DS_ERR_WORKSPACE;
+  return ds::launch_lmhead_confidence(hidden, weight, rows, hid, V, ld_h, ld_w, conf, tok, workspace, status,
+                                      reinterpret_cast<cudaStream_t>(stream));
+}
+
 int ds_confidence_static(const void *logits, int32_t dtype, int64_t rows, int64_t V, int64_t ld,
                          const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok, void *stream) {
   if (dtype != DS_F32 && dtype != DS_BF16) return DS_ERR_INVALID_ARG;

@@ -53,9 +53,12 @@
 #include <mutex>
 
 #include "ds_common.cuh"
+#include "ds_sm100.cuh"
 
 namespace ds {
 namespace {
+
+using namespace sm100;
 
 // Optional timeline of CTA 0 (build with -DDS_TRACE): SM clock at a few points of every role's loop.
 #ifdef DS_TRACE
@@ -82,7 +85,6 @@ constexpr int kXRows = 16;                  // N of the transposed problem (the 
 constexpr int kXMax = 8;                    // extra rows actually served
 constexpr int kXChunkBytes = kXRows * 128;
 constexpr int kIdxCap = 2048;               // entries of a shared index list kept in shared memory
-constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 constexpr float kXLimit = 24.0f;            // log2 units a transposed score may exceed its reference by
 
@@ -127,177 +129,6 @@ struct TcParams {
   int n_items;       // B * Hkv * n_mtiles
   float scale_log2;  // softmax scale * log2(e)
 };
-
-// ------------------------------------------------------------------------------------------------
-// PTX wrappers
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false when it gave up (or another role already did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (it > 128) {
-      __nanosleep(64);
-      if (*abort_flag) return false;
-    }
-  }
-  *abort_flag = 1;
-  return false;
-}
-// Bounded wait for two barriers at once (their polls overlap instead of adding up).
-__device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b,
-                                           volatile int *abort_flag) {
-  bool a = false, b = false;
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (!a) a = mbar_try_wait(bar_a, parity_a);
-    if (!b) b = mbar_try_wait(bar_b, parity_b);
-    if (a && b) return true;
-    if (it > 128) {
-      __nanosleep(64);
-      if (*abort_flag) return false;
-    }
-  }
-  *abort_flag = 1;
-  return false;
-}
-
-// True in exactly one lane of the (converged) warp.
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "elect.sync _|p, 0xffffffff;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(pred));
-  return pred != 0;
-}
-
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
-      : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-
-// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate.
-__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                        uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]: A is M x 16, one row per lane, two bf16 per 32-bit column.
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                        uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// mbarrier arrives once all MMAs issued so far by this thread have completed.
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// 16 lanes x 32 columns twice: threads 0-15 get columns taddr.., threads 16-31 the same 16 lanes at
-// columns taddr + kSplit...
-template <int kSplit>
-__device__ __forceinline__ void tmem_ld16x2_32(uint32_t taddr, uint32_t *r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x32bx2.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32], %33;"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr), "n"(kSplit)
-      : "memory");
-}
-template <int kSplit>
-__device__ __forceinline__ void tmem_st16x2_32(uint32_t taddr, const uint32_t *r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.16x32bx2.x32.b32 [%32], %33, "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
-      ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
-        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
-        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr), "n"(kSplit)
-      : "memory");
-}
-// 32 lanes x 8 columns: thread t gets columns taddr .. taddr + 7 of lane t of the warp's quadrant.
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t *r) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t *r) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};" ::"r"(r[0]), "r"(r[1]),
-               "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(taddr)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128.
-__host__ __device__ constexpr uint32_t instr_desc(int n, bool a_mn_major, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
-         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-__device__ __forceinline__ float fmax3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
 
 // ------------------------------------------------------------------------------------------------
 // Producer helper: fetch n gathered rows (logical rows R0 .. R0+n-1 of a stacked sequence whose
@@ -590,8 +421,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     // ============================ MMA issuer: S = Q K^T ============================
     // The whole warp walks the loop (uniform control flow keeps descriptors in uniform registers);
     // one elected lane issues the MMAs and commits.
-    constexpr uint32_t idesc_qk = instr_desc(kBlockN, false, false);
-    constexpr uint32_t idesc_qk_x = instr_desc(kXRows, false, false);  // S_x^T = K Q_x^T
+    constexpr uint32_t idesc_qk = instr_desc(kBlockM, kBlockN, false, false);
+    constexpr uint32_t idesc_qk_x = instr_desc(kBlockM, kXRows, false, false);  // S_x^T = K Q_x^T
     const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
     // descriptors of byte 0 of each operand region; a K-step only adds to the address field
     const uint64_t dq = smem_desc(sbase + G_::kOffQ, 16, 1024);
@@ -662,8 +493,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     timed_out = !ok;
   } else if (warp == kPvWarp) {
     // ============================ MMA issuer: O += P V ============================
-    constexpr uint32_t idesc_pv = instr_desc(D, false, true);
-    constexpr uint32_t idesc_pv_x = instr_desc(kXRows, true, false);  // O_x^T = V^T P_x^T
+    constexpr uint32_t idesc_pv = instr_desc(kBlockM, D, false, true);
+    constexpr uint32_t idesc_pv_x = instr_desc(kBlockM, kXRows, true, false);  // O_x^T = V^T P_x^T
     const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
     const uint64_t dpx = smem_desc(sbase + G_::kOffPx, 16, 1024);
     const uint64_t dv0 = smem_desc(sbase + G_::kOffRing, kChunkBytes, 1024);  // V tile, MN-major
@@ -1044,25 +875,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
-using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                              const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn encode_fn() {
-  static EncodeFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void *p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeFn>(p);
-    else
-      (void)cudaGetLastError();
-  });
-  return fn;
-}
-
 // [B][H][rows][D] bf16 tensor with element strides {batch, head, row}; box = 64 columns x box_rows rows.
 bool make_map(CUtensorMap *m, const void *base, int D, long long rows, int H, int B, const int64_t stride[3], int box_rows) {
   EncodeFn fn = encode_fn();
@@ -1126,6 +938,23 @@ int launch_d(const ds_attn_params &p, cudaStream_t stream) {
 }
 
 }  // namespace
+
+namespace sm100 {
+EncodeFn encode_fn() {
+  static EncodeFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeFn>(p);
+    else
+      (void)cudaGetLastError();
+  });
+  return fn;
+}
+}  // namespace sm100
 
 #ifdef DS_TRACE
 extern "C" __attribute__((visibility("default"))) int ds_debug_trace(long long *host_out) {

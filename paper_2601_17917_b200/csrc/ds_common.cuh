@@ -45,6 +45,10 @@ size_t confidence_workspace_bytes(int64_t rows, int64_t V, int dtype);
 int launch_confidence_static(const void *logits, int dtype, int64_t rows, int64_t V, int64_t ld,
                              const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
                              cudaStream_t stream);
+size_t lmhead_workspace_bytes(int64_t rows, int64_t V);
+int launch_lmhead_confidence(const void *hidden, const void *weight, int64_t rows, int64_t hid, int64_t V, int64_t ld_h,
+                             int64_t ld_w, float *conf, int32_t *tok, void *workspace, uint32_t *status,
+                             cudaStream_t stream);
 int launch_select(const ds_select_params &p, cudaStream_t stream);
 int launch_attn_simt(const ds_attn_params &p, cudaStream_t stream);
 int launch_attn_tc(const ds_attn_params &p, cudaStream_t stream);

@@ -168,3 +168,23 @@ def uniform_confidences(cfg: StepConfig, eos_id: int, eos_p: float = 0.05, step:
     plant = torch.rand(cfg.B, cfg.K, generator=g) < eos_p
     tok[plant] = eos_id
     return conf, tok
+
+
+def lmhead_inputs(cfg: StepConfig, hid: int, device="cpu", rows: int | None = None, V: int | None = None):
+    """Inputs of the fused output projection: hidden [rows, hid] ~ N(0,1) and an output embedding
+    weight [V, hid] ~ N(0, 4/hid), so that the logits hidden @ weight.T are ~ N(0, 2^2) like the stored
+    logits of ``logits``.  A seeded Bernoulli(spike_p) subset of rows gets the spike: the embedding of a
+    seeded token is moved along that row's hidden vector so that its logit rises by about ``spike``."""
+    rows = cfg.rows if rows is None else rows
+    V = cfg.V if V is None else V
+    s = cfg.seed + 400
+    h = _normal((rows, hid), s, device, torch.float32)
+    w = _normal((V, hid), s + 1, device, torch.float32, std=2.0 / hid ** 0.5)
+    g = _gen(s + 2, "cpu")
+    is_spiked = torch.rand(rows, generator=g) < cfg.spike_p
+    col = torch.randint(0, V, (rows,), generator=g)
+    r = torch.nonzero(is_spiked).flatten().to(h.device)
+    if r.numel():
+        hr = h[r]
+        w[col[r.cpu()].to(h.device)] += float(cfg.spike) * hr / (hr * hr).sum(1, keepdim=True)
+    return h.to(torch.bfloat16), w.to(torch.bfloat16)
