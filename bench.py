@@ -374,6 +374,47 @@ class OracleSample:
         return full, t3 - t0
 
 
+HIDDEN_SIZE = {126464: 4096, 152064: 3584}   # hidden size of the model a vocabulary size belongs to
+
+
+def time_lmhead(cfg, device, reps=10):
+    """The widened path: output projection fused with Eq. 4 (ds_lmhead_confidence), timed alone with CUDA
+    events, and the unfused alternative (library GEMM writing bf16 logits + ds_confidence) beside it."""
+    import torch
+    import paper_2601_17917_b200 as ds
+    from paper_2601_17917_b200 import workloads as wl
+    hid = HIDDEN_SIZE.get(cfg.V, 4096)
+    h, w = wl.lmhead_inputs(cfg, hid, device=device)
+    rows, V = cfg.rows, cfg.V
+    ws = torch.empty(max(ds.ds_lmhead_confidence_workspace(rows, V), 256), dtype=torch.uint8, device=device)
+    conf = torch.empty(rows, dtype=torch.float32, device=device)
+    tok = torch.empty(rows, dtype=torch.int32, device=device)
+    z = torch.empty(rows, V, dtype=torch.bfloat16, device=device)
+    cws = torch.empty(max(ds.ds_confidence_workspace(rows, V, torch.bfloat16), 256), dtype=torch.uint8, device=device)
+
+    def fused():
+        ds.ds_lmhead_confidence(h, w, conf=conf, tok=tok, workspace=ws)
+
+    def unfused():
+        torch.matmul(h, w.T, out=z)
+        ds.ds_confidence(z, conf=conf, tok=tok, workspace=cws)
+
+    out = {}
+    for name, fn in (("fused", fused), ("unfused", unfused)):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        out[name] = a.elapsed_time(b) / reps
+    flops = 2.0 * rows * hid * V
+    return out, flops, hid, V * hid * 2 + rows * hid * 2
+
+
 def run_reference(args, cfg):
     if int(os.environ.get("RANK", "0")) != 0:
         return
@@ -411,8 +452,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-lmhead", action="store_true", help="skip the extra timing of ds_lmhead_confidence")
     ap.add_argument("--stages", default="attn,confidence,select",
                     help="comma list of the stages a step runs (profiling a single kernel)")
+    ap.add_argument("--vocab", type=int, default=0, help="override the vocabulary size (small profiler cases)")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the batch size of the configuration (small cases for profiler captures)")
     args = ap.parse_args()
@@ -421,6 +464,8 @@ def main():
     cfg = wl.CONFIGS[args.config]
     if args.batch > 0:
         cfg = wl.shrink(cfg, B=args.batch, name=f"{cfg.name}-B{args.batch}")
+    if args.vocab > 0:
+        cfg = wl.shrink(cfg, V=args.vocab, name=f"{cfg.name}-V{args.vocab}")
     if args.impl == "reference":
         run_reference(args, cfg)
         return
@@ -444,6 +489,12 @@ def main():
         if world > 1:
             dist.barrier()
 
+    if args.stages == "lmhead":            # profiling run of the widened kernel alone
+        t, flops, hid, in_bytes = time_lmhead(cfg, device, reps=max(1, args.steps))
+        print(json.dumps({"stages": "lmhead", "config": {"workload": cfg.name, "rows": cfg.rows, "hidden": hid, "V": cfg.V},
+                          "ms": t["fused"], "tflops": flops / (t["fused"] * 1e-3) / 1e12, "unfused_ms": t["unfused"]}),
+              flush=True)
+        return
     warmup = max(args.warmup, 3)
     # replicas: every rank draws its own batch (its rank offsets the seed); no data-path collective
     rcfg = rank_config(cfg, rank)
@@ -512,6 +563,19 @@ def main():
         line["stages"] = args.stages          # partial step: a profiling run, not a bench value
     if e2e:
         line["e2e"] = e2e
+    if not args.no_lmhead and args.stages == "attn,confidence,select":
+        del step
+        torch.cuda.empty_cache()
+        t, flops, hid, in_bytes = time_lmhead(cfg, device)
+        tf = flops / (t["fused"] * 1e-3) / 1e12
+        line["lmhead_confidence"] = {
+            "what": "output projection fused with Eq. 4 (logits never stored); not part of `value`",
+            "rows": cfg.rows, "hidden": hid, "V": cfg.V, "ms": t["fused"],
+            "roofline": {"kernel": "ds_lmhead_confidence", "bound": "tensor", "achieved": tf, "peak": pk["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": tf / pk["bf16_tflops"], "peak_source": pk["_source"] + " (burst)",
+                         "traffic": None},
+            "weight_stream_gbs": in_bytes / (t["fused"] * 1e-3) / 1e9,
+            "unfused_ms": t["unfused"], "unfused": "torch.matmul (library GEMM) to bf16 logits + ds_confidence"}
     if not args.no_cpu_baseline and world == 1:
         smp = OracleSample(cfg, 32, 128)
         full_s, spent = smp.time()
