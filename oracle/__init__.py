@@ -14,6 +14,9 @@ Contents
   tail over prefix + whole tail, materialising every score row.  It exists to
   pin ``attn``: retaining every suffix position must reproduce it.
 * ``confidence`` (C, ``oracle_confidence``): Eq. 4.
+* ``rope_gather`` (C, ``oracle_rope_gather``): rotary encoding of the retained
+  rows with their original position ids (Eq. 7's "positional information ...
+  via RoPE position IDs") and their gather into compact Q/K/V.
 * ``lmhead_confidence`` (C, ``oracle_lmhead_confidence``): the output projection
   (last of the "remaining model components" that turn attention outputs into
   logits) composed with Eq. 4, logits kept in float64.
@@ -67,6 +70,9 @@ def _load():
         lib.oracle_lmhead_confidence.restype = ctypes.c_int
         lib.oracle_lmhead_confidence.argtypes = [c_fp, c_fp, ctypes.c_long, ctypes.c_long, ctypes.c_long, c_dp,
                                                  c_ip, c_dp]
+        lib.oracle_rope_gather.restype = ctypes.c_int
+        lib.oracle_rope_gather.argtypes = [c_fp, c_fp, c_fp] + [ctypes.c_int] * 6 + [
+            c_ip, ctypes.c_long, ctypes.c_long, ctypes.c_double, c_dp, c_dp, c_dp]
         lib.oracle_threshold.restype = ctypes.c_float
         lib.oracle_threshold.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_float,
                                          ctypes.c_float]
@@ -190,6 +196,26 @@ def confidence(logits):
     if rc != 0:
         raise ValueError("oracle_confidence rejected its arguments")
     return conf, tok
+
+
+def rope_gather(q_raw, k_raw, v_raw, idx, pos_offset, theta=10000.0):
+    """Rotary encoding (rotate-half pairing) of the retained tail rows with their original position ids
+    ``pos_offset + idx[i]`` and gather into compact buffers.  q_raw [B,Hq,T,D]; k_raw, v_raw [B,Hkv,T,D];
+    idx [Lq] or [B,Lq].  Returns float64 (q [B,Hq,Lq,D], k [B,Hkv,Lq,D], v [B,Hkv,Lq,D])."""
+    lib = _load()
+    q_raw, k_raw, v_raw = map(_f32, (q_raw, k_raw, v_raw))
+    B, Hq, T, D = q_raw.shape
+    Hkv = k_raw.shape[1]
+    assert k_raw.shape == (B, Hkv, T, D) and v_raw.shape == (B, Hkv, T, D)
+    idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
+    Lq, bstride = (idx.shape[0], 0) if idx.ndim == 1 else (idx.shape[1], idx.shape[1])
+    q = np.empty((B, Hq, Lq, D)); k = np.empty((B, Hkv, Lq, D)); v = np.empty((B, Hkv, Lq, D))
+    rc = lib.oracle_rope_gather(_ptr(q_raw, ctypes.c_float), _ptr(k_raw, ctypes.c_float), _ptr(v_raw, ctypes.c_float),
+                                B, Hq, Hkv, D, T, Lq, _ptr(idx, ctypes.c_int32), bstride, int(pos_offset), float(theta),
+                                _ptr(q, ctypes.c_double), _ptr(k, ctypes.c_double), _ptr(v, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("oracle_rope_gather rejected its arguments")
+    return q, k, v
 
 
 def lmhead_confidence(hidden, weight, want_logits=False):

@@ -281,3 +281,62 @@ int oracle_lmhead_confidence(const float *hidden, const float *weight, long rows
   }
   return bad ? -2 : 0;
 }
+
+/*
+ * Rotary position encoding of the retained rows with their ORIGINAL position
+ * ids, and their gather into compact buffers (Method, "Attenuation Guided
+ * Suffix Modeling": the pruned suffix keeps "the logical ordering of tokens
+ * via RoPE position IDs"; Eq. 7 names the retained set, Eq. 8 the pruned input).
+ *
+ * For every batch b, head h and retained row i (tail row r = idx[i], absolute
+ * position p = pos_offset + r), with half = D / 2 and, for d < half,
+ * angle = p * theta^(-2 d / D):
+ *     out[d]        = x[d] cos(angle) - x[d + half] sin(angle)
+ *     out[d + half] = x[d + half] cos(angle) + x[d] sin(angle)
+ * (the "rotate half" pairing of dimension d with d + D/2).  Q and K are
+ * rotated, V is only gathered.
+ *
+ *   q_raw           [B][Hq ][T][D]   float32 (bf16 widened exactly)
+ *   k_raw, v_raw    [B][Hkv][T][D]
+ *   idx             [Lq] (idx_bstride 0) or [B][Lq]
+ *   q_out           [B][Hq ][Lq][D]  double
+ *   k_out, v_out    [B][Hkv][Lq][D]  double
+ */
+int oracle_rope_gather(const float *q_raw, const float *k_raw, const float *v_raw,
+                       int B, int Hq, int Hkv, int D, int T, int Lq,
+                       const int32_t *idx, long idx_bstride, long pos_offset,
+                       double theta, double *q_out, double *k_out, double *v_out) {
+  if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || (D & 1) || T < 0 || Lq < 0 || theta <= 0.0) return -1;
+  const int half = D / 2;
+  for (int b = 0; b < B; ++b)
+    for (int i = 0; i < Lq; ++i) {
+      const int r = idx[(long)b * idx_bstride + i];
+      if (r < 0 || r >= T) return -1;
+    }
+  for (int b = 0; b < B; ++b)
+    for (int i = 0; i < Lq; ++i) {
+      const int r = idx[(long)b * idx_bstride + i];
+      const double p = (double)(pos_offset + r);
+      for (int which = 0; which < 2; ++which) {       /* 0: queries, 1: keys */
+        const int H = which ? Hkv : Hq;
+        const float *src = which ? k_raw : q_raw;
+        double *dst = which ? k_out : q_out;
+        for (int h = 0; h < H; ++h) {
+          const float *x = src + (((long)b * H + h) * T + r) * D;
+          double *o = dst + (((long)b * H + h) * Lq + i) * D;
+          for (int d = 0; d < half; ++d) {
+            const double angle = p * pow(theta, -2.0 * (double)d / (double)D);
+            const double c = cos(angle), s = sin(angle);
+            o[d] = (double)x[d] * c - (double)x[d + half] * s;
+            o[d + half] = (double)x[d + half] * c + (double)x[d] * s;
+          }
+        }
+      }
+      for (int h = 0; h < Hkv; ++h) {
+        const float *x = v_raw + (((long)b * Hkv + h) * T + r) * D;
+        double *o = v_out + (((long)b * Hkv + h) * Lq + i) * D;
+        for (int d = 0; d < D; ++d) o[d] = (double)x[d];
+      }
+    }
+  return 0;
+}
