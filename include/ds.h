@@ -144,6 +144,52 @@ DS_API int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_
                   void *workspace, size_t workspace_bytes, void *stream);
 
 /* ------------------------------------------------------------------------
+ * ds_rope_gather  (Eq. 7 position ids, Eq. 8 pruned input, prefix-cache append)
+ *
+ * The suffix pruning keeps "the logical ordering of tokens via RoPE position
+ * IDs": a retained row keeps the position it has in the full sequence.  This
+ * entry point takes the un-rotated projections of the whole tail and produces
+ * what ds_attn_pruned consumes, compact and rotated.  For every batch b and
+ * retained row i (tail row r = idx[i], absolute position pos = pos_offset + r):
+ *     q_out[b][h][i] = rope(q_raw[b][h][r], pos)      (all Hq heads)
+ *     k_out[b][g][i] = rope(k_raw[b][g][r], pos)      (all Hkv heads)
+ *     v_out[b][g][i] = v_raw[b][g][r]
+ * rope pairs dimension d with d + D/2 ("rotate half"):
+ *     out[d]       = x[d] cos(a_d) - x[d + D/2] sin(a_d)
+ *     out[d + D/2] = x[d + D/2] cos(a_d) + x[d] sin(a_d),   a_d = pos * rope_theta^(-2d/D)
+ * ds_attn_pruned is then called on the compact buffers with T = Lq and
+ * idx = 0 .. Lq-1.  When n_append > 0 the first n_append retained rows (the
+ * current block, once it is finished) are also written to the prefix cache at
+ * rows cache_row0 .. cache_row0 + n_append - 1 (rotated K, plain V).
+ *
+ * All tensors bf16, D contiguous, D a multiple of 16, element strides for
+ * batch / head / row, bases and strides 16-byte aligned.  Out-of-range idx
+ * entries are clamped and flagged (DS_DEV_INDEX) like in ds_attn_pruned.
+ * ------------------------------------------------------------------------ */
+typedef struct {
+  int32_t B, Hq, Hkv, D;
+  int32_t T;                          /* rows of the raw tail buffers */
+  int32_t Lq;                         /* retained rows */
+  const void *q_raw;                  /* [B][Hq ][T][D] */
+  const void *k_raw, *v_raw;          /* [B][Hkv][T][D] */
+  int64_t q_stride[3], kv_stride[3];
+  const int32_t *idx;                 /* [Lq] or [B][Lq] */
+  int64_t idx_batch_stride;
+  int32_t pos_offset;                 /* absolute position of tail row 0 (= prefix length) */
+  float rope_theta;                   /* frequency base, > 1 */
+  void *q_out;                        /* [B][Hq ][Lq][D] */
+  void *k_out, *v_out;                /* [B][Hkv][Lq][D] */
+  int64_t q_out_stride[3], kv_out_stride[3];
+  void *k_cache, *v_cache;            /* optional [B][Hkv][rows][D]; needed when n_append > 0 */
+  int64_t cache_stride[3];
+  int32_t cache_row0, n_append;
+  uint32_t *status;                   /* optional device word */
+} ds_rope_params;
+
+/* `p` is a HOST pointer; the pointers inside it are device pointers. */
+DS_API int ds_rope_gather(const ds_rope_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
  * ds_lmhead_confidence  (output projection + Eq. 4, fused)
  *
  * In the prediction forward the attention outputs are "processed by the

@@ -19,7 +19,7 @@ from . import workloads  # noqa: F401  (seeded synthetic inputs)
 __all__ = [
     "lib", "retained_indices", "ds_attn_pruned", "ds_attn_pruned_workspace", "ds_confidence",
     "ds_confidence_workspace", "ds_confidence_static", "ds_lmhead_confidence", "ds_lmhead_confidence_workspace",
-    "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
+    "ds_rope_gather", "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
     "ds_launch_count", "DsError", "DS_F32", "DS_BF16", "DS_DEV_INDEX", "DS_DEV_TIMEOUT",
 ]
 
@@ -49,6 +49,21 @@ class _AttnParams(ctypes.Structure):
         ("idx", ctypes.c_void_p), ("idx_batch_stride", ctypes.c_int64), ("scale", ctypes.c_float),
         ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t), ("status", ctypes.c_void_p),
+    ]
+
+
+class _RopeParams(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32),
+        ("T", ctypes.c_int32), ("Lq", ctypes.c_int32),
+        ("q_raw", ctypes.c_void_p), ("k_raw", ctypes.c_void_p), ("v_raw", ctypes.c_void_p),
+        ("q_stride", ctypes.c_int64 * 3), ("kv_stride", ctypes.c_int64 * 3),
+        ("idx", ctypes.c_void_p), ("idx_batch_stride", ctypes.c_int64),
+        ("pos_offset", ctypes.c_int32), ("rope_theta", ctypes.c_float),
+        ("q_out", ctypes.c_void_p), ("k_out", ctypes.c_void_p), ("v_out", ctypes.c_void_p),
+        ("q_out_stride", ctypes.c_int64 * 3), ("kv_out_stride", ctypes.c_int64 * 3),
+        ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p), ("cache_stride", ctypes.c_int64 * 3),
+        ("cache_row0", ctypes.c_int32), ("n_append", ctypes.c_int32), ("status", ctypes.c_void_p),
     ]
 
 
@@ -82,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.ds_confidence.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.ds_rope_gather.restype = ctypes.c_int
+        L.ds_rope_gather.argtypes = [ctypes.POINTER(_RopeParams), ctypes.c_void_p]
         L.ds_lmhead_confidence_workspace.restype = ctypes.c_size_t
         L.ds_lmhead_confidence_workspace.argtypes = [ctypes.c_int64, ctypes.c_int64]
         L.ds_lmhead_confidence.restype = ctypes.c_int
@@ -242,6 +259,56 @@ def ds_confidence(logits, row_list=None, conf=None, tok=None, workspace=None, st
     if rc != DS_OK:
         raise DsError(rc, "ds_confidence")
     return conf, tok
+
+
+def ds_rope_gather(q_raw, k_raw, v_raw, idx, pos_offset, rope_theta=10000.0, q_out=None, k_out=None, v_out=None,
+                   k_cache=None, v_cache=None, cache_row0=0, n_append=0, status=None, stream=None):
+    """Rotary encoding of the retained tail rows with their original position ids and gather into compact
+    buffers (Eq. 7-8); optionally appends the first ``n_append`` retained rows to the prefix cache.
+    q_raw [B,Hq,T,D]; k_raw, v_raw [B,Hkv,T,D] bf16; idx int32 [Lq] or [B,Lq].  Returns (q, k, v) compact
+    [B,H,Lq,D], ready for ``ds_attn_pruned`` with ``idx = arange(Lq)``."""
+    _check_dev(q_raw, k_raw, v_raw, idx, q_out, k_out, v_out, k_cache, v_cache, status)
+    B, Hq, T, D = q_raw.shape
+    Hkv = k_raw.shape[1]
+    Lq = idx.shape[-1]
+    for t in (q_raw, k_raw, v_raw):
+        if t.dtype != torch.bfloat16 or t.stride(-1) != 1:
+            raise ValueError("inputs must be bf16 with a contiguous head dimension")
+    if k_raw.stride() != v_raw.stride():
+        raise ValueError("K and V must share strides")
+    if idx.dtype != torch.int32:
+        raise TypeError("idx must be int32")
+    dev = q_raw.device
+    if q_out is None:
+        q_out = torch.empty((B, Hq, Lq, D), dtype=torch.bfloat16, device=dev)
+    if k_out is None:
+        k_out = torch.empty((B, Hkv, Lq, D), dtype=torch.bfloat16, device=dev)
+    if v_out is None:
+        v_out = torch.empty((B, Hkv, Lq, D), dtype=torch.bfloat16, device=dev)
+    if k_out.stride() != v_out.stride():
+        raise ValueError("k_out and v_out must share strides")
+    p = _RopeParams()
+    p.B, p.Hq, p.Hkv, p.D, p.T, p.Lq = B, Hq, Hkv, D, T, Lq
+    p.q_raw, p.k_raw, p.v_raw = q_raw.data_ptr(), k_raw.data_ptr(), v_raw.data_ptr()
+    p.q_stride[:] = q_raw.stride()[:3]
+    p.kv_stride[:] = k_raw.stride()[:3]
+    p.idx = idx.data_ptr()
+    p.idx_batch_stride = 0 if idx.dim() == 1 else idx.stride(0)
+    p.pos_offset, p.rope_theta = int(pos_offset), float(rope_theta)
+    p.q_out, p.k_out, p.v_out = q_out.data_ptr(), k_out.data_ptr(), v_out.data_ptr()
+    p.q_out_stride[:] = q_out.stride()[:3]
+    p.kv_out_stride[:] = k_out.stride()[:3]
+    if n_append:
+        if k_cache is None or v_cache is None or k_cache.stride() != v_cache.stride():
+            raise ValueError("appending needs k_cache and v_cache with equal strides")
+        p.k_cache, p.v_cache = k_cache.data_ptr(), v_cache.data_ptr()
+        p.cache_stride[:] = k_cache.stride()[:3]
+    p.cache_row0, p.n_append = int(cache_row0), int(n_append)
+    p.status = status.data_ptr() if status is not None else None
+    rc = lib().ds_rope_gather(ctypes.byref(p), _stream(stream))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_rope_gather")
+    return q_out, k_out, v_out
 
 
 def ds_lmhead_confidence_workspace(rows: int, V: int) -> int:

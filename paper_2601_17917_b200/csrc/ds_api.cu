@@ -114,6 +114,30 @@ int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_t V, in
                                workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
+int ds_rope_gather(const ds_rope_params *p, void *stream) {
+  if (!p) return DS_ERR_INVALID_ARG;
+  if (p->B < 0 || p->Hq <= 0 || p->Hkv <= 0 || p->D <= 0 || p->T <= 0 || p->Lq < 0 || p->Lq > p->T) return DS_ERR_INVALID_ARG;
+  if (p->pos_offset < 0 || !(p->rope_theta > 1.0f) || p->n_append < 0 || p->n_append > p->Lq || p->cache_row0 < 0)
+    return DS_ERR_INVALID_ARG;
+  if (p->D % 16 != 0) return DS_ERR_UNSUPPORTED;
+  if (p->B == 0 || p->Lq == 0) return DS_OK;
+  if (!p->q_raw || !p->k_raw || !p->v_raw || !p->idx || !p->q_out || !p->k_out || !p->v_out) return DS_ERR_INVALID_ARG;
+  if (p->n_append > 0 && (!p->k_cache || !p->v_cache)) return DS_ERR_INVALID_ARG;
+  if (p->idx_batch_stride != 0 && p->idx_batch_stride < p->Lq) return DS_ERR_INVALID_ARG;
+  const void *ptrs[] = {p->q_raw, p->k_raw, p->v_raw, p->q_out, p->k_out, p->v_out, p->n_append ? p->k_cache : nullptr,
+                        p->n_append ? p->v_cache : nullptr};
+  for (const void *q : ptrs)
+    if (q && !ds::aligned(q, 16)) return DS_ERR_INVALID_ARG;
+  const int64_t *strides[] = {p->q_stride, p->kv_stride, p->q_out_stride, p->kv_out_stride, p->cache_stride};
+  for (int k = 0; k < 5; ++k) {
+    if (k == 4 && p->n_append == 0) continue;
+    for (int d = 0; d < 3; ++d)
+      if (strides[k][d] < 0 || strides[k][d] % 8 != 0) return DS_ERR_INVALID_ARG;
+    if (strides[k][2] < p->D) return DS_ERR_INVALID_ARG;
+  }
+  return ds::launch_rope_gather(*p, reinterpret_cast<cudaStream_t>(stream));
+}
+
 size_t ds_lmhead_confidence_workspace(int64_t rows, int64_t V) { return ds::lmhead_workspace_bytes(rows, V); }
 
 int ds_lmhead_confidence(const void *hidden, const void *weight, int64_t rows, int64_t hid, int64_t V, int64_t ld_h,

@@ -50,6 +50,7 @@ int launch_lmhead_confidence(const void *hidden, const void *weight, int64_t row
                              int64_t ld_w, float *conf, int32_t *tok, void *workspace, uint32_t *status,
                              cudaStream_t stream);
 int launch_select(const ds_select_params &p, cudaStream_t stream);
+int launch_rope_gather(const ds_rope_params &p, cudaStream_t stream);
 int launch_attn_simt(const ds_attn_params &p, cudaStream_t stream);
 int launch_attn_tc(const ds_attn_params &p, cudaStream_t stream);
 bool attn_tc_supported(const ds_attn_params &p);

@@ -47,12 +47,17 @@ int main(void) {
   printf("%zu %zu %zu %zu %zu\n", sizeof(ds_select_params), offsetof(ds_select_params, tau0),
          offsetof(ds_select_params, seq_list), offsetof(ds_select_params, n_seq_dev),
          offsetof(ds_select_params, active_cnt));
+  printf("%zu %zu %zu %zu %zu %zu\n", sizeof(ds_rope_params), offsetof(ds_rope_params, q_stride),
+         offsetof(ds_rope_params, idx), offsetof(ds_rope_params, rope_theta), offsetof(ds_rope_params, k_cache),
+         offsetof(ds_rope_params, status));
   return 0;
 }''')
     exe = tmp_path / "layout"
     subprocess.run(["gcc", "-I", str(ROOT / "include"), str(src), "-o", str(exe)], check=True)
-    a, s = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.strip().splitlines()
-    A, S = ds._AttnParams, ds._SelectParams
+    a, s, r = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.strip().splitlines()
+    A, S, R = ds._AttnParams, ds._SelectParams, ds._RopeParams
+    assert [int(v) for v in r.split()] == [ctypes.sizeof(R), R.q_stride.offset, R.idx.offset, R.rope_theta.offset,
+                                           R.k_cache.offset, R.status.offset]
     assert [int(v) for v in a.split()] == [ctypes.sizeof(A), A.q_stride.offset, A.idx.offset, A.scale.offset,
                                            A.out.offset, A.status.offset]
     assert [int(v) for v in s.split()] == [ctypes.sizeof(S), S.tau0.offset, S.seq_list.offset,
