@@ -415,6 +415,35 @@ def time_lmhead(cfg, device, reps=10):
     return out, flops, hid, V * hid * 2 + rows * hid * 2
 
 
+def time_rope(cfg, device, reps=20):
+    """The widened path: rotary encoding + gather of the retained rows (ds_rope_gather), timed alone."""
+    import torch
+    import paper_2601_17917_b200 as ds
+    from paper_2601_17917_b200 import workloads as wl
+    x = wl.attention_inputs(cfg, device=device)
+    idx = torch.tensor(ds.retained_indices(cfg.gen, cfg.K, 0, cfg.w, cfg.keep_last), dtype=torch.int32, device=device)
+    Lq = idx.numel()
+    qo = torch.empty((cfg.B, cfg.Hq, Lq, cfg.D), dtype=torch.bfloat16, device=device)
+    ko = torch.empty((cfg.B, cfg.Hkv, Lq, cfg.D), dtype=torch.bfloat16, device=device)
+    vo = torch.empty_like(ko)
+
+    def fn():
+        ds.ds_rope_gather(x["q_tail"], x["k_tail"], x["v_tail"], idx, cfg.P, 10000.0, q_out=qo, k_out=ko, v_out=vo)
+
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    nbytes = 2 * cfg.B * (cfg.Hq + 2 * cfg.Hkv) * Lq * cfg.D * 2       # every retained row read once, written once
+    return ms, nbytes
+
+
 def run_reference(args, cfg):
     if int(os.environ.get("RANK", "0")) != 0:
         return
@@ -495,6 +524,11 @@ def main():
                           "ms": t["fused"], "tflops": flops / (t["fused"] * 1e-3) / 1e12, "unfused_ms": t["unfused"]}),
               flush=True)
         return
+    if args.stages == "rope":              # profiling run of the widened kernel alone
+        ms, nbytes = time_rope(cfg, device, reps=max(1, args.steps))
+        print(json.dumps({"stages": "rope", "config": {"workload": cfg.name}, "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9}),
+              flush=True)
+        return
     warmup = max(args.warmup, 3)
     # replicas: every rank draws its own batch (its rank offsets the seed); no data-path collective
     rcfg = rank_config(cfg, rank)
@@ -565,6 +599,12 @@ def main():
         line["e2e"] = e2e
     if not args.no_lmhead and args.stages == "attn,confidence,select":
         del step
+        torch.cuda.empty_cache()
+        r_ms, r_bytes = time_rope(cfg, device)
+        line["rope_gather"] = {"what": "rotary encoding + gather of the retained rows; not part of `value`", "ms": r_ms,
+                               "roofline": {"kernel": "ds_rope_gather", "bound": "hbm", "achieved": r_bytes / (r_ms * 1e-3) / 1e9,
+                                            "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": r_bytes / (r_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                                            "algorithmic_bytes": r_bytes, "traffic": None, "peak_source": pk["_source"]}}
         torch.cuda.empty_cache()
         t, flops, hid, in_bytes = time_lmhead(cfg, device)
         tf = flops / (t["fused"] * 1e-3) / 1e12
