@@ -58,12 +58,13 @@ int validate_attn(const ds_attn_params *p) {
   return DS_OK;
 }
 
-enum class AttnPath { kAuto, kSimt, kTc };
+enum class AttnPath { kAuto, kSimt, kTc, kTc2 };
 AttnPath forced_path() {
   const char *e = std::getenv("DS_ATTN_PATH");
   if (!e) return AttnPath::kAuto;
   if (!std::strcmp(e, "simt")) return AttnPath::kSimt;
   if (!std::strcmp(e, "tc")) return AttnPath::kTc;
+  if (!std::strcmp(e, "tc2")) return AttnPath::kTc2;
   return AttnPath::kAuto;
 }
 
@@ -85,7 +86,8 @@ int ds_attn_pruned(const ds_attn_params *p, void *stream) {
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const ds::AttnPath path = ds::forced_path();
   const bool tc_ok = ds::attn_tc_supported(*p);
-  if (path == ds::AttnPath::kTc && !tc_ok) return DS_ERR_UNSUPPORTED;
+  if ((path == ds::AttnPath::kTc || path == ds::AttnPath::kTc2) && !tc_ok) return DS_ERR_UNSUPPORTED;
+  if (tc_ok && path == ds::AttnPath::kTc2) return ds::launch_attn_tc2(*p, st);
   if (tc_ok && path != ds::AttnPath::kSimt) {
     const size_t need = ds::attn_tc_workspace_bytes(*p);
     if (need > 0 && (!p->workspace || !ds::aligned(p->workspace, 256) || p->workspace_bytes < need))

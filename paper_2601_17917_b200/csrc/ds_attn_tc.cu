@@ -52,6 +52,7 @@
 #include <cstring>
 #include <mutex>
 
+#include "ds_attn_tiles.cuh"
 #include "ds_common.cuh"
 #include "ds_sm100.cuh"
 
@@ -59,6 +60,7 @@ namespace ds {
 namespace {
 
 using namespace sm100;
+using namespace attn;
 
 // Optional timeline of CTA 0 (build with -DDS_TRACE): SM clock at a few points of every role's loop.
 #ifdef DS_TRACE
@@ -73,18 +75,14 @@ __device__ long long g_trace[4][256][8];
   } while (0)
 #endif
 
-constexpr int kBlockM = 128;
-constexpr int kBlockN = 128;
 constexpr int kSoftmaxWarps = 8;
 constexpr int kXWarps = 4;  // softmax of the transposed problem (one per TMEM lane quadrant)
 constexpr int kNumThreads = (kSoftmaxWarps + 3 + kXWarps) * 32;
 constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1, kXWarp0 = kSoftmaxWarps + 2;
 constexpr int kPvWarp = kXWarp0 + kXWarps;  // second MMA issuer
-constexpr int kChunkBytes = 128 * 128;      // one [128 rows][64 bf16] swizzled chunk
 constexpr int kXRows = 16;                  // N of the transposed problem (the smallest N for M = 128)
 constexpr int kXMax = 8;                    // extra rows actually served
 constexpr int kXChunkBytes = kXRows * 128;
-constexpr int kIdxCap = 2048;               // entries of a shared index list kept in shared memory
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 constexpr float kXLimit = 24.0f;            // log2 units a transposed score may exceed its reference by
 
@@ -115,80 +113,11 @@ struct Geo {
 static_assert(Geo<128>::kSmemBytes <= 227 * 1024, "shared memory budget");
 static_assert(Geo<64>::kSmemBytes <= 227 * 1024, "shared memory budget");
 
-struct TcParams {
-  CUtensorMap kpre, vpre, k32, k1, v32, v1, q32, q1;
-  const int32_t *idx;
-  long long idx_bstride;
-  void *out;
-  long long out_stride[3];
-  float *lse;
-  uint32_t *status;
-  int B, Hq, Hkv, G, P, T, Lq;
-  int n_mtiles;      // M-tiles per (batch, KV head)
-  int x_rows;        // extra rows riding with the last M-tile (0 = none)
-  int n_items;       // B * Hkv * n_mtiles
-  float scale_log2;  // softmax scale * log2(e)
+struct TcParams : attn::AttnCommon {
+  int n_mtiles;  // M-tiles per (batch, KV head)
+  int x_rows;    // extra rows riding with the last M-tile (0 = none)
+  int n_items;   // B * Hkv * n_mtiles
 };
-
-// ------------------------------------------------------------------------------------------------
-// Producer helper: fetch n gathered rows (logical rows R0 .. R0+n-1 of a stacked sequence whose
-// period is Lq) into a swizzled tile whose 64-column chunks are chunk_stride bytes apart.  The whole
-// warp calls it; lane 0 issues the copies.  Returns the bytes issued (valid on lane 0).
-// ------------------------------------------------------------------------------------------------
-template <int D>
-__device__ __forceinline__ uint32_t gather_rows(const TcParams &prm, const CUtensorMap *map32, const CUtensorMap *map1,
-                                                uint32_t dst, uint32_t chunk_stride, uint32_t bar, int R0, int n,
-                                                int head0, int b, int32_t *idx_s, const int32_t *idx_cache,
-                                                bool &bad_index, bool staged = false) {
-  const int lane = threadIdx.x & 31;
-  const int Lq = prm.Lq;
-  // position of logical row R0 inside its head; divisions only when the stacking actually wraps
-  int head = head0, pos0 = R0;
-  if (pos0 >= Lq) {
-    head += pos0 / Lq;
-    pos0 %= Lq;
-  }
-  __syncwarp();
-  if (!staged) {  // otherwise idx_s already holds these rows (the K tile of the same rows came first)
-    const int32_t *ix = prm.idx + (long long)b * prm.idx_bstride;
-    for (int r = lane; r < n; r += 32) {
-      int pos = pos0 + r;
-      if (pos >= Lq) pos %= Lq;
-      int v;
-      if (idx_cache != nullptr && pos < kIdxCap) {
-        v = idx_cache[pos];  // validated when it was cached
-      } else {
-        v = ix[pos];
-        if (v < 0 || v >= prm.T) {
-          bad_index = true;
-          v = v < 0 ? 0 : prm.T - 1;
-        }
-      }
-      idx_s[r] = v;
-    }
-    __syncwarp();
-  }
-  uint32_t bytes = 0;
-  if (lane == 0) {
-    int r = 0, pos = pos0;
-    while (r < n) {
-      const int row = idx_s[r];
-      const bool box32 = ((r & 7) == 0) && (r + 32 <= n) && (pos + 32 <= Lq) && (idx_s[r + 31] - row == 31);
-      const int step = box32 ? 32 : 1;
-#pragma unroll
-      for (int c = 0; c < Geo<D>::kChunks; ++c)
-        tma_load_4d(dst + c * chunk_stride + r * 128, box32 ? map32 : map1, bar, c * 64, row, head, b);
-      bytes += (uint32_t)step * 128u * Geo<D>::kChunks;
-      r += step;
-      pos += step;
-      if (pos >= Lq) {  // a 32-row box never crosses a head, so this is at most one wrap
-        pos -= Lq;
-        ++head;
-      }
-    }
-  }
-  return bytes;
-}
 
 struct Item {
   int b, hk, mt, m_rows, x_rows;
@@ -875,47 +804,13 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
-// [B][H][rows][D] bf16 tensor with element strides {batch, head, row}; box = 64 columns x box_rows rows.
-bool make_map(CUtensorMap *m, const void *base, int D, long long rows, int H, int B, const int64_t stride[3], int box_rows) {
-  EncodeFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)H, (cuuint64_t)B};
-  // a dimension of extent 1 may carry any stride; keep them valid multiples of 16 bytes
-  const cuuint64_t strides[3] = {(cuuint64_t)stride[2] * 2, (cuuint64_t)(H > 1 ? stride[1] : stride[2] * rows) * 2,
-                                 (cuuint64_t)(B > 1 ? stride[0] : (H > 1 ? stride[1] * H : stride[2] * rows)) * 2};
-  const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int D>
 int launch_d(const ds_attn_params &p, cudaStream_t stream) {
   // the attribute is per device: set it at every launch (cheap)
   DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes));
   TcParams prm;
   memset(&prm, 0, sizeof(prm));
-  bool ok = true;
-  if (p.P > 0) {
-    ok = ok && make_map(&prm.kpre, p.k_prefix, D, p.P, p.Hkv, p.B, p.kv_prefix_stride, kBlockN);
-    ok = ok && make_map(&prm.vpre, p.v_prefix, D, p.P, p.Hkv, p.B, p.kv_prefix_stride, kBlockN);
-  }
-  ok = ok && make_map(&prm.k32, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 32);
-  ok = ok && make_map(&prm.k1, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 1);
-  ok = ok && make_map(&prm.v32, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 32);
-  ok = ok && make_map(&prm.v1, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 1);
-  ok = ok && make_map(&prm.q32, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 32);
-  ok = ok && make_map(&prm.q1, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 1);
-  if (!ok) return DS_ERR_CUDA;
-  prm.idx = p.idx;
-  prm.idx_bstride = p.idx_batch_stride;
-  prm.out = p.out;
-  for (int k = 0; k < 3; ++k) prm.out_stride[k] = p.out_stride[k];
-  prm.lse = p.lse;
-  prm.status = p.status;
-  prm.B = p.B, prm.Hq = p.Hq, prm.Hkv = p.Hkv, prm.G = p.Hq / p.Hkv, prm.P = p.P, prm.T = p.T, prm.Lq = p.Lq;
-  prm.scale_log2 = p.scale * kLog2e;
+  if (!fill_common(prm, p)) return DS_ERR_CUDA;
   // stacked query rows of one KV head: full 128-row tiles, and a remainder that either rides along
   // with the last full tile (1..kXMax rows, D = 128) or gets a tile of its own
   const long long rows_total = (long long)prm.G * p.Lq;
@@ -938,6 +833,51 @@ int launch_d(const ds_attn_params &p, cudaStream_t stream) {
 }
 
 }  // namespace
+
+namespace attn {
+namespace {
+// [B][H][rows][D] bf16 tensor with element strides {batch, head, row}; box = 64 columns x box_rows rows.
+bool make_map(CUtensorMap *m, const void *base, int D, long long rows, int H, int B, const int64_t stride[3], int box_rows) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)H, (cuuint64_t)B};
+  // a dimension of extent 1 may carry any stride; keep them valid multiples of 16 bytes
+  const cuuint64_t strides[3] = {(cuuint64_t)stride[2] * 2, (cuuint64_t)(H > 1 ? stride[1] : stride[2] * rows) * 2,
+                                 (cuuint64_t)(B > 1 ? stride[0] : (H > 1 ? stride[1] * H : stride[2] * rows)) * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool fill_common(AttnCommon &c, const ds_attn_params &p) {
+  const int D = p.D;
+  bool ok = true;
+  if (p.P > 0) {
+    ok = ok && make_map(&c.kpre, p.k_prefix, D, p.P, p.Hkv, p.B, p.kv_prefix_stride, kBlockN);
+    ok = ok && make_map(&c.vpre, p.v_prefix, D, p.P, p.Hkv, p.B, p.kv_prefix_stride, kBlockN);
+  }
+  ok = ok && make_map(&c.k32, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 32);
+  ok = ok && make_map(&c.k1, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 1);
+  ok = ok && make_map(&c.v32, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 32);
+  ok = ok && make_map(&c.v1, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 1);
+  ok = ok && make_map(&c.q32, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 32);
+  ok = ok && make_map(&c.q1, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 1);
+  if (!ok) return false;
+  c.idx = p.idx;
+  c.idx_bstride = p.idx_batch_stride;
+  c.out = p.out;
+  for (int k = 0; k < 3; ++k) c.out_stride[k] = p.out_stride[k];
+  c.lse = p.lse;
+  c.status = p.status;
+  c.B = p.B, c.Hq = p.Hq, c.Hkv = p.Hkv, c.G = p.Hq / p.Hkv, c.P = p.P, c.T = p.T, c.Lq = p.Lq;
+  c.scale_log2 = p.scale * kLog2e;
+  return true;
+}
+}  // namespace attn
 
 namespace sm100 {
 EncodeFn encode_fn() {

@@ -1,0 +1,94 @@
+// Pieces shared by the tensor-core attention kernels: the launch parameters common to both, the gather
+// of index-listed rows into swizzled shared-memory tiles, and the tensor-map encoding of the
+// [B][H][rows][D] operands.
+#pragma once
+#include "ds_sm100.cuh"
+
+namespace ds {
+namespace attn {
+
+using namespace sm100;
+
+constexpr int kBlockM = 128;
+constexpr int kBlockN = 128;
+constexpr int kChunkBytes = 128 * 128;  // one [128 rows][64 bf16] swizzled chunk
+constexpr int kIdxCap = 2048;           // entries of a shared index list kept in shared memory
+
+struct AttnCommon {
+  CUtensorMap kpre, vpre, k32, k1, v32, v1, q32, q1;
+  const int32_t *idx;
+  long long idx_bstride;
+  void *out;
+  long long out_stride[3];
+  float *lse;
+  uint32_t *status;
+  int B, Hq, Hkv, G, P, T, Lq;
+  float scale_log2;  // softmax scale * log2(e)
+};
+
+// ------------------------------------------------------------------------------------------------
+// Producer helper: fetch n gathered rows (logical rows R0 .. R0+n-1 of a stacked sequence whose
+// period is Lq) into a swizzled tile whose 64-column chunks are chunk_stride bytes apart.  The whole
+// warp calls it; lane 0 issues the copies.  Returns the bytes issued (valid on lane 0).
+// ------------------------------------------------------------------------------------------------
+template <int D>
+__device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUtensorMap *map32, const CUtensorMap *map1,
+                                                uint32_t dst, uint32_t chunk_stride, uint32_t bar, int R0, int n,
+                                                int head0, int b, int32_t *idx_s, const int32_t *idx_cache,
+                                                bool &bad_index, bool staged = false) {
+  const int lane = threadIdx.x & 31;
+  const int Lq = prm.Lq;
+  // position of logical row R0 inside its head; divisions only when the stacking actually wraps
+  int head = head0, pos0 = R0;
+  if (pos0 >= Lq) {
+    head += pos0 / Lq;
+    pos0 %= Lq;
+  }
+  __syncwarp();
+  if (!staged) {  // otherwise idx_s already holds these rows (the K tile of the same rows came first)
+    const int32_t *ix = prm.idx + (long long)b * prm.idx_bstride;
+    for (int r = lane; r < n; r += 32) {
+      int pos = pos0 + r;
+      if (pos >= Lq) pos %= Lq;
+      int v;
+      if (idx_cache != nullptr && pos < kIdxCap) {
+        v = idx_cache[pos];  // validated when it was cached
+      } else {
+        v = ix[pos];
+        if (v < 0 || v >= prm.T) {
+          bad_index = true;
+          v = v < 0 ? 0 : prm.T - 1;
+        }
+      }
+      idx_s[r] = v;
+    }
+    __syncwarp();
+  }
+  uint32_t bytes = 0;
+  if (lane == 0) {
+    int r = 0, pos = pos0;
+    while (r < n) {
+      const int row = idx_s[r];
+      const bool box32 = ((r & 7) == 0) && (r + 32 <= n) && (pos + 32 <= Lq) && (idx_s[r + 31] - row == 31);
+      const int step = box32 ? 32 : 1;
+#pragma unroll
+      for (int c = 0; c < (D / 64); ++c)
+        tma_load_4d(dst + c * chunk_stride + r * 128, box32 ? map32 : map1, bar, c * 64, row, head, b);
+      bytes += (uint32_t)step * 128u * (D / 64);
+      r += step;
+      pos += step;
+      if (pos >= Lq) {  // a 32-row box never crosses a head, so this is at most one wrap
+        pos -= Lq;
+        ++head;
+      }
+    }
+  }
+  return bytes;
+}
+
+
+// Fills the tensor maps and the fields common to both kernels from the C-ABI parameters.
+bool fill_common(AttnCommon &c, const ds_attn_params &p);
+
+}  // namespace attn
+}  // namespace ds

@@ -53,6 +53,7 @@ int launch_select(const ds_select_params &p, cudaStream_t stream);
 int launch_rope_gather(const ds_rope_params &p, cudaStream_t stream);
 int launch_attn_simt(const ds_attn_params &p, cudaStream_t stream);
 int launch_attn_tc(const ds_attn_params &p, cudaStream_t stream);
+int launch_attn_tc2(const ds_attn_params &p, cudaStream_t stream);
 bool attn_tc_supported(const ds_attn_params &p);
 size_t attn_tc_workspace_bytes(const ds_attn_params &p);
 
