@@ -92,6 +92,10 @@ int ds_attn_pruned(const ds_attn_params *p, void *stream) {
     const size_t need = ds::attn_tc_workspace_bytes(*p);
     if (need > 0 && (!p->workspace || !ds::aligned(p->workspace, 256) || p->workspace_bytes < need))
       return DS_ERR_WORKSPACE;
+    // Many M-tiles per KV head (the unpruned reference, a cache-refresh step): the two-tile kernel shares every
+    // KV tile between two M-tiles; measured faster from about 8 tile pairs on, slower below.
+    const long long stacked_rows = (long long)(p->Hq / p->Hkv) * p->Lq;
+    if (path == ds::AttnPath::kAuto && stacked_rows >= 2048) return ds::launch_attn_tc2(*p, st);
     return ds::launch_attn_tc(*p, st);
   }
   return ds::launch_attn_simt(*p, st);

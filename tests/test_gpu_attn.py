@@ -127,6 +127,22 @@ def test_many_items_per_cta():
     _run_small(40, 8, 4, 128, 300, 300, list(range(256)) + [299], torch.bfloat16, seed=80)  # 2 tiles + 2 extra rows
 
 
+@pytest.mark.parametrize("path", ["tc", "tc2"])
+def test_both_tensor_core_kernels_on_the_same_shapes(path, monkeypatch):
+    """The one-tile and the two-tile kernel are chosen by shape; here each is forced on shapes of both kinds
+    (several M-tiles per KV head, a single partial tile, GQA stacking, D = 64, no prefix, peaked scores)."""
+    monkeypatch.setenv("DS_ATTN_PATH", path)
+    T = 300
+    _run_small(2, 2, 2, 128, 300, T, list(range(256)) + [T - 1], torch.bfloat16, seed=31)
+    _run_small(1, 14, 2, 128, 512, T, list(range(96)) + [T - 1], torch.bfloat16, seed=32)
+    _run_small(2, 4, 4, 128, 1000, 400, list(range(320)) + [399], torch.bfloat16, seed=33, q_scale=2.0)
+    _run_small(1, 2, 2, 64, 200, T, list(range(T)), torch.bfloat16, seed=34)
+    _run_small(3, 8, 2, 128, 0, 200, list(range(129)) + [199], torch.bfloat16, seed=35)
+    _run_small(40, 8, 4, 128, 300, T, list(range(256)) + [T - 1], torch.bfloat16, seed=36)
+    _run_small(1, 2, 2, 128, 130, 200, list(range(63)) + [199], torch.bfloat16, seed=37, q_scale=3.0)
+    _run_small(1, 2, 2, 128, 700, 200, list(range(128)) + [199], torch.bfloat16, seed=38, q_scale=3.0, k_boost=(300, 5.0))
+
+
 def test_scattered_and_per_batch_index_lists():
     rng = np.random.default_rng(3)
     T, B = 500, 3
