@@ -285,14 +285,16 @@ def time_resident(step, steps, warmup, sampler, barrier):
     return total_ms, stage_ms, launches, windows, extra
 
 
-def time_e2e(cfg, device, steps, warmup):
+def time_e2e(cfg, device, steps, warmup, cache_resident=False):
     """Same step from pinned host buffers: H2D of everything the step reads, the three calls,
-    D2H of the results, all inside the timed region."""
+    D2H of the results, all inside the timed region.  ``cache_resident``: the prefix KV cache stays on
+    the device (the method computes it once per block and reuses it at every step); only what changes
+    from step to step is copied."""
     import torch
     dev_step = Step(cfg, device, compact_tail=True)
     host_in, dev_in = [], []
     for x in dev_step.layers:
-        for k in ("q_tail", "k_tail", "v_tail", "k_pre", "v_pre"):
+        for k in ("q_tail", "k_tail", "v_tail") + (() if cache_resident else ("k_pre", "v_pre")):
             dev_in.append(x[k])
     dev_in += [dev_step.logits, dev_step.x_block, dev_step.masked, dev_step.idx]
     for t in dev_in:
@@ -555,6 +557,11 @@ def main():
         e2e = {"value": job_throughput(world, e_ms), "unit": "steps/s", "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "ms_per_step": e_ms, "steps": e2e_steps,
                "layout": "tail rows shipped compact (T = Lq): only what the step reads crosses the link"}
+        # second figure: the prefix KV cache resident, as it is between the steps of a block
+        r_ms, r_h2d, r_d2h = time_e2e(rcfg, device, e2e_steps, 3, cache_resident=True)
+        r_ms = max_over_ranks(r_ms, world, device)
+        e2e["prefix_cache_resident"] = {"value": job_throughput(world, r_ms), "unit": "steps/s", "ms_per_step": r_ms,
+                                        "h2d_bytes_per_step": int(r_h2d), "d2h_bytes_per_step": int(r_d2h)}
 
     if rank != 0:
         if world > 1:
