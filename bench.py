@@ -14,7 +14,7 @@ ds_unmask_select over one batch of seeded synthetic input.  Prints ONE JSON line
 * ``e2e``: the same step through the public API starting from pinned HOST
   buffers: host->device copies of everything the step reads and device->host
   copies of its results are inside the timed region.
-* ``cpu_baseline``: the CPU oracle, as it stands, timed on this machine's host
+* ``cpu_baseline``: the CPU oracle, as it stands, timed on the machine's host
   cores on a bounded sample of the same workload and scaled to a full step.
 * ``--impl reference`` times that oracle as the main line.
 """
@@ -37,7 +37,7 @@ DEFAULT_CONFIG = "long32-w64"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes; None until a capture of that kernel and workload exists)
 NCU_TRAFFIC: dict = {
-    # captured on the batch-4 instance of the workload (profiles/*-B4.md) and scaled by the items one launch
+    # captured on the batch-4 instance of the workload (the committed ncu summaries) and scaled by the items one launch
     # processes (x8: traffic is proportional to the rows streamed); set back to None when a kernel changes
     "long32-w64": {"attn_bytes_per_launch": 8 * (282.50e6 + 7.26e6), "confidence_bytes_per_launch": 8 * (64.78e6 + 0.33e6)},
 }
