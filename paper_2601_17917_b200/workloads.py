@@ -75,6 +75,10 @@ CONFIGS: dict[str, StepConfig] = {
                               keep_last=True, dtype="bf16", V=126464, spike_p=0.5, seed=5000),
     "long32-all": StepConfig("long32-all", B=32, Hq=32, Hkv=32, D=128, P=4096, gen=4096, K=64, w=-1,
                              keep_last=True, dtype="bf16", V=126464, spike_p=0.5, seed=5000),
+    # the first step of a block ("cache refresh"): every position of the sequence is a query, nothing is cached yet;
+    # prompt 1024 + generation 1024 rows, all retained -> dense bidirectional attention, bound by the tensor cores
+    "refresh8": StepConfig("refresh8", B=8, Hq=32, Hkv=32, D=128, P=0, gen=2048, K=32, w=-1,
+                           keep_last=True, dtype="bf16", V=126464, spike_p=0.5, seed=6000),
 }
 
 

@@ -257,3 +257,8 @@ def test_full_size_llada_batched_layers():
 def test_full_size_unpruned_reference_sampled_rows():
     # "all 4032": the window covers the whole suffix; Lq = 4096, Lkv = 8192
     _sampled_parity(wl.CONFIGS["long32-all"], n_slices=4, q_rows=16)
+
+
+def test_cache_refresh_step_dense_no_prefix():
+    # first step of a block: no cached prefix, every row of the sequence is a query and a key (Lq = Lkv = 2048)
+    _sampled_parity(wl.CONFIGS["refresh8"], n_slices=4, q_rows=16)
