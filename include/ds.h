@@ -115,6 +115,15 @@ typedef struct {
   void *workspace;
   size_t workspace_bytes;
   uint32_t *status;                  /* optional device word, DS_DEV_* bits are OR-ed in */
+  /* Optional restriction to some sequences (e.g. ds_unmask_select's active_seq: the sequences whose block
+   * still has masked positions).  seq_list = n_seq ascending batch numbers in [0, B); NULL = all B (n_seq and
+   * n_seq_dev are then ignored).  n_seq_dev, when not NULL, is a device scalar read by the kernel that
+   * overrides n_seq as the count (clamped to [0, n_seq]; n_seq then only sizes the launch), so that a loop
+   * over steps needs no host synchronisation.  Outputs of sequences not listed are left untouched; a listed
+   * number outside [0, B) sets DS_DEV_INDEX and is clamped. */
+  const int32_t *seq_list;
+  int32_t n_seq;
+  const int32_t *n_seq_dev;
 } ds_attn_params;
 
 /* HOST, pure: bytes of workspace ds_attn_pruned needs for *p (0 when none). */
@@ -142,6 +151,13 @@ DS_API size_t ds_confidence_workspace(int64_t rows, int64_t V, int32_t dtype);
 DS_API int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_t V, int64_t ld,
                   const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
                   void *workspace, size_t workspace_bytes, void *stream);
+/* The same with the length of row_list held on the device: `n_listed_dev` (device scalar, not NULL) is read
+ * by the kernel and clamped to [0, n_listed_max]; n_listed_max sizes the launch; the workspace is that of
+ * ds_confidence (ds_confidence_workspace(rows, V, dtype)).  A listed row outside [0, rows) is skipped.  Meant for ds_unmask_select's masked_rows /
+ * masked_cnt: Eq. 4 is only needed at the positions that are still masked, and the count changes every step. */
+DS_API int ds_confidence_listed(const void *logits, int32_t dtype, int64_t rows, int64_t V, int64_t ld,
+                         const int32_t *row_list, int64_t n_listed_max, const int32_t *n_listed_dev,
+                         float *conf, int32_t *tok, void *workspace, size_t workspace_bytes, void *stream);
 
 /* ------------------------------------------------------------------------
  * ds_rope_gather  (Eq. 7 position ids, Eq. 8 pruned input, prefix-cache append)
@@ -268,6 +284,9 @@ DS_API int ds_confidence_static(const void *logits, int32_t dtype, int64_t rows,
  *     eos_exit[b]  |= 1 when an accepted token equals eos_id with conf >= eos_tau
  *     active_seq    = ascending list of processed sequences with block_done == 0,
  *                     *active_cnt its length
+ *     masked_rows   = (optional) ascending list of b * K + i over the processed sequences b and the positions i
+ *                     that are still masked after the step, *masked_cnt its length: the rows of a
+ *                     [B * K][V] logit matrix the next step needs Eq. 4 for
  * ratio_extra = 0 counts the block only; ratio_extra = R also counts the
  * retained suffix rows of the query (all still masked).  alpha = 0 gives the
  * fixed-threshold rule.  eos_id < 0 disables the early-exit flag.
@@ -296,6 +315,8 @@ typedef struct {
   uint8_t *eos_exit;            /* [B] in/out */
   int32_t *active_seq;          /* [B] */
   int32_t *active_cnt;          /* [1] */
+  int32_t *masked_rows;         /* optional [B*K] */
+  int32_t *masked_cnt;          /* [1], needed with masked_rows */
 } ds_select_params;
 
 /* `p` is a HOST pointer; the pointers inside it are device pointers. */

@@ -49,6 +49,7 @@ class _AttnParams(ctypes.Structure):
         ("idx", ctypes.c_void_p), ("idx_batch_stride", ctypes.c_int64), ("scale", ctypes.c_float),
         ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t), ("status", ctypes.c_void_p),
+        ("seq_list", ctypes.c_void_p), ("n_seq", ctypes.c_int32), ("n_seq_dev", ctypes.c_void_p),
     ]
 
 
@@ -75,7 +76,7 @@ class _SelectParams(ctypes.Structure):
         ("eos_tau", ctypes.c_float), ("seq_list", ctypes.c_void_p), ("n_seq", ctypes.c_int32),
         ("n_seq_dev", ctypes.c_void_p), ("sel_idx", ctypes.c_void_p), ("sel_cnt", ctypes.c_void_p),
         ("block_done", ctypes.c_void_p), ("eos_exit", ctypes.c_void_p), ("active_seq", ctypes.c_void_p),
-        ("active_cnt", ctypes.c_void_p),
+        ("active_cnt", ctypes.c_void_p), ("masked_rows", ctypes.c_void_p), ("masked_cnt", ctypes.c_void_p),
     ]
 
 
@@ -97,6 +98,11 @@ def lib() -> ctypes.CDLL:
         L.ds_confidence.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.ds_confidence_listed.restype = ctypes.c_int
+        L.ds_confidence_listed.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                           ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                                           ctypes.c_void_p]
         L.ds_rope_gather.restype = ctypes.c_int
         L.ds_rope_gather.argtypes = [ctypes.POINTER(_RopeParams), ctypes.c_void_p]
         L.ds_lmhead_confidence_workspace.restype = ctypes.c_size_t
@@ -173,7 +179,8 @@ def retained_indices(gen_len: int, K: int, c: int, w_tokens: int, keep_last: boo
     return idx
 
 
-def _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status):
+def _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status,
+                 seq_list=None, n_seq=None, n_seq_dev=None):
     B, Hq, T, D = q_tail.shape
     Hkv = k_tail.shape[1]
     P = 0 if k_prefix is None else k_prefix.shape[2]
@@ -204,6 +211,14 @@ def _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, ls
     p.workspace = workspace.data_ptr() if workspace is not None else None
     p.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     p.status = status.data_ptr() if status is not None else None
+    if seq_list is not None:
+        if seq_list.dtype != torch.int32 or (n_seq_dev is not None and n_seq_dev.dtype != torch.int32):
+            raise TypeError("seq_list and n_seq_dev must be int32")
+        if seq_list.numel() == 0:
+            raise ValueError("seq_list must have room for at least one entry (use n_seq=0 for an empty list)")
+        p.seq_list = seq_list.data_ptr()
+        p.n_seq = seq_list.numel() if n_seq is None else min(int(n_seq), seq_list.numel())
+        p.n_seq_dev = n_seq_dev.data_ptr() if n_seq_dev is not None else None
     return p
 
 
@@ -213,15 +228,18 @@ def ds_attn_pruned_workspace(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, sc
 
 
 def ds_attn_pruned(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out=None, lse=None,
-                   workspace=None, status=None, stream=None):
+                   workspace=None, status=None, stream=None, seq_list=None, n_seq=None, n_seq_dev=None):
     """Pruned attention (Eq. 7-8).  q_tail [B,Hq,T,D]; k_tail, v_tail [B,Hkv,T,D];
     k_prefix, v_prefix [B,Hkv,P,D] or None; idx int32 [Lq] or [B,Lq] on the device.
+    seq_list (int32, ascending batch numbers; its first n_seq entries, or as many as the device scalar
+    n_seq_dev says) restricts the call to those sequences.
     Returns ``out`` [B,Hq,Lq,D].  Allocates ``out``/``workspace`` with torch when not given."""
-    _check_dev(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, out, lse, workspace, status)
+    _check_dev(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, out, lse, workspace, status, seq_list, n_seq_dev)
     B, Hq, T, D = q_tail.shape
     if out is None:
         out = torch.empty((B, Hq, idx.shape[-1], D), dtype=q_tail.dtype, device=q_tail.device)
-    p = _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status)
+    p = _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status,
+                     seq_list, n_seq, n_seq_dev)
     if workspace is None:
         need = int(lib().ds_attn_pruned_workspace(ctypes.byref(p)))
         if need:
@@ -258,6 +276,27 @@ def ds_confidence(logits, row_list=None, conf=None, tok=None, workspace=None, st
                              _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
     if rc != DS_OK:
         raise DsError(rc, "ds_confidence")
+    return conf, tok
+
+
+def ds_confidence_listed(logits, row_list, n_listed_dev, conf, tok, n_listed_max=None, workspace=None, stream=None):
+    """Eq. 4 over the first ``*n_listed_dev`` rows named in ``row_list`` (both on the device, int32), e.g.
+    ds_unmask_select's masked_rows / masked_cnt.  conf/tok [rows] are updated at those rows only."""
+    _check_dev(logits, row_list, n_listed_dev, conf, tok, workspace)
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits must be [rows, V] with contiguous rows")
+    if row_list.dtype != torch.int32 or n_listed_dev.dtype != torch.int32:
+        raise TypeError("row_list and n_listed_dev must be int32")
+    rows, V = logits.shape
+    n_max = min(rows, row_list.numel()) if n_listed_max is None else int(n_listed_max)
+    if workspace is None:
+        need = ds_confidence_workspace(rows, V, logits.dtype)
+        workspace = torch.empty(max(need, 1), dtype=torch.uint8, device=logits.device)
+    rc = lib().ds_confidence_listed(_ptr(logits), _dtype_code(logits), rows, V, logits.stride(0), _ptr(row_list),
+                                    n_max, _ptr(n_listed_dev), _ptr(conf), _ptr(tok), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_confidence_listed")
     return conf, tok
 
 
@@ -368,7 +407,8 @@ def ds_unmask_select(conf, tok, masked, x_block, tau0, alpha, ratio_extra=0, eos
                      seq_list=None, n_seq=None, n_seq_dev=None, out=None, stream=None):
     """Eq. 9-10 selection step.  conf f32 [B,K], tok i32 [B,K]; masked u8 [B,K] and
     x_block i32 [B,K] are updated in place.  Returns a dict of device tensors:
-    sel_idx, sel_cnt, block_done, eos_exit, active_seq, active_cnt (pass ``out`` to reuse them)."""
+    sel_idx, sel_cnt, block_done, eos_exit, active_seq, active_cnt, masked_rows, masked_cnt
+    (pass ``out`` to reuse them; masked_rows/masked_cnt are written when ``out`` holds them)."""
     _check_dev(conf, tok, masked, x_block, seq_list, n_seq_dev)
     B, K = conf.shape
     dev = conf.device
@@ -381,7 +421,9 @@ def ds_unmask_select(conf, tok, masked, x_block, tau0, alpha, ratio_extra=0, eos
                    block_done=torch.zeros(B, dtype=torch.uint8, device=dev),
                    eos_exit=torch.zeros(B, dtype=torch.uint8, device=dev),
                    active_seq=torch.empty(max(B, 1), dtype=torch.int32, device=dev),
-                   active_cnt=torch.zeros(1, dtype=torch.int32, device=dev))
+                   active_cnt=torch.zeros(1, dtype=torch.int32, device=dev),
+                   masked_rows=torch.empty(max(B * K, 1), dtype=torch.int32, device=dev),
+                   masked_cnt=torch.zeros(1, dtype=torch.int32, device=dev))
     p = _SelectParams()
     p.B, p.K = B, K
     p.conf, p.tok, p.masked, p.x_block = conf.data_ptr(), tok.data_ptr(), masked.data_ptr(), x_block.data_ptr()
@@ -396,6 +438,8 @@ def ds_unmask_select(conf, tok, masked, x_block, tau0, alpha, ratio_extra=0, eos
     p.sel_idx, p.sel_cnt = out["sel_idx"].data_ptr(), out["sel_cnt"].data_ptr()
     p.block_done, p.eos_exit = out["block_done"].data_ptr(), out["eos_exit"].data_ptr()
     p.active_seq, p.active_cnt = out["active_seq"].data_ptr(), out["active_cnt"].data_ptr()
+    if out.get("masked_rows") is not None:
+        p.masked_rows, p.masked_cnt = out["masked_rows"].data_ptr(), out["masked_cnt"].data_ptr()
     rc = lib().ds_unmask_select(ctypes.byref(p), _stream(stream))
     if rc != DS_OK:
         raise DsError(rc, "ds_unmask_select")

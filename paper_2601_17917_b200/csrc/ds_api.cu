@@ -37,6 +37,9 @@ int validate_attn(const ds_attn_params *p) {
   if (p->P > 0 && (!p->k_prefix || !p->v_prefix)) return DS_ERR_INVALID_ARG;
   if (p->idx_batch_stride != 0 && p->idx_batch_stride < p->Lq) return DS_ERR_INVALID_ARG;
   if (!(p->scale == p->scale)) return DS_ERR_INVALID_ARG;
+  if (p->seq_list && (p->n_seq < 0 || p->n_seq > p->B || !aligned(p->seq_list, 4) ||
+                      (p->n_seq_dev && !aligned(p->n_seq_dev, 4))))
+    return DS_ERR_INVALID_ARG;
   const int64_t unit = (p->dtype == DS_BF16) ? 8 : 4;  // 16 bytes
   const void *ptrs[] = {p->q_tail, p->k_tail, p->v_tail, p->out, p->P > 0 ? p->k_prefix : nullptr,
                         p->P > 0 ? p->v_prefix : nullptr};
@@ -116,7 +119,22 @@ int ds_confidence(const void *logits, int32_t dtype, int64_t rows, int64_t V, in
   const size_t esz = dtype == DS_BF16 ? 2 : 4;
   if (!ds::aligned(logits, esz) || !ds::aligned(conf, 4) || !ds::aligned(tok, 4)) return DS_ERR_INVALID_ARG;
   if (row_list && (n_listed < 0 || n_listed > rows)) return DS_ERR_INVALID_ARG;
-  return ds::launch_confidence(logits, dtype, rows, V, ld, row_list, n_listed, conf, tok, workspace,
+  return ds::launch_confidence(logits, dtype, rows, V, ld, row_list, n_listed, nullptr, conf, tok, workspace,
+                               workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int ds_confidence_listed(const void *logits, int32_t dtype, int64_t rows, int64_t V, int64_t ld,
+                         const int32_t *row_list, int64_t n_listed_max, const int32_t *n_listed_dev, float *conf,
+                         int32_t *tok, void *workspace, size_t workspace_bytes, void *stream) {
+  if (dtype != DS_F32 && dtype != DS_BF16) return DS_ERR_INVALID_ARG;
+  if (rows < 0 || V <= 0 || ld < V || V > 0x7fffffffLL) return DS_ERR_INVALID_ARG;
+  if (!row_list || !n_listed_dev || n_listed_max < 0 || n_listed_max > rows) return DS_ERR_INVALID_ARG;
+  if (rows == 0 || n_listed_max == 0) return DS_OK;
+  if (!logits || !conf || !tok) return DS_ERR_INVALID_ARG;
+  const size_t esz = dtype == DS_BF16 ? 2 : 4;
+  if (!ds::aligned(logits, esz) || !ds::aligned(conf, 4) || !ds::aligned(tok, 4) || !ds::aligned(n_listed_dev, 4))
+    return DS_ERR_INVALID_ARG;
+  return ds::launch_confidence(logits, dtype, rows, V, ld, row_list, n_listed_max, n_listed_dev, conf, tok, workspace,
                                workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
@@ -186,6 +204,8 @@ int ds_unmask_select(const ds_select_params *p, void *stream) {
     return DS_ERR_INVALID_ARG;
   if (p->seq_list && (p->n_seq < 0 || p->n_seq > p->B)) return DS_ERR_INVALID_ARG;
   if (!p->seq_list && p->n_seq_dev) return DS_ERR_INVALID_ARG;
+  if (p->masked_rows && !p->masked_cnt) return DS_ERR_INVALID_ARG;
+  if ((long long)p->B * p->K > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   return ds::launch_select(*p, reinterpret_cast<cudaStream_t>(stream));
 }
 

@@ -49,11 +49,22 @@ __global__ void __launch_bounds__(kRowsPerCta * 32) attn_simt_kernel(const ds_at
   const int lane = threadIdx.x & 31;
   const int i = blockIdx.x * kRowsPerCta + (threadIdx.x >> 5);
   if (i >= p.Lq) return;
-  const int hq = blockIdx.y, b = blockIdx.z;
+  const int hq = blockIdx.y;
+  int b = blockIdx.z;
+  bool bad_index = false;
+  if (p.seq_list != nullptr) {  // blockIdx.z counts listed sequences
+    int n = p.n_seq;
+    if (p.n_seq_dev != nullptr) n = max(0, min(n, *p.n_seq_dev));
+    if (b >= n) return;
+    b = p.seq_list[b];
+    if (b < 0 || b >= p.B) {
+      bad_index = true;
+      b = b < 0 ? 0 : p.B - 1;
+    }
+  }
   const int hk = hq / (p.Hq / p.Hkv);
   const int32_t *ix = p.idx + (long long)b * p.idx_batch_stride;
   const int dofs = lane * DPL;
-  bool bad_index = false;
 
   auto tail_row = [&](int j) {
     int r = ix[j];
@@ -143,7 +154,9 @@ __global__ void __launch_bounds__(kRowsPerCta * 32) attn_simt_kernel(const ds_at
 
 template <typename T>
 int launch_t(const ds_attn_params &p, cudaStream_t stream) {
-  const dim3 grid(ceil_div(p.Lq, kRowsPerCta), p.Hq, p.B);
+  const int n_seq = p.seq_list ? p.n_seq : p.B;
+  if (n_seq == 0) return DS_OK;
+  const dim3 grid(ceil_div(p.Lq, kRowsPerCta), p.Hq, n_seq);
   const dim3 block(kRowsPerCta * 32);
   switch (p.D / 32) {
     case 1: attn_simt_kernel<T, 1><<<grid, block, 0, stream>>>(p); break;

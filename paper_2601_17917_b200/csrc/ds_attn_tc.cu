@@ -127,7 +127,7 @@ __device__ __forceinline__ Item decode_item(const TcParams &prm, int item) {
   it.mt = item % prm.n_mtiles;
   const int bh = item / prm.n_mtiles;
   it.hk = bh % prm.Hkv;
-  it.b = bh / prm.Hkv;
+  it.b = attn::listed_batch(prm, bh / prm.Hkv);
   const int rows_total = prm.G * prm.Lq;
   it.x_rows = (it.mt == prm.n_mtiles - 1) ? prm.x_rows : 0;
   it.m_rows = min(kBlockM, rows_total - it.x_rows - it.mt * kBlockM);
@@ -203,11 +203,14 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_base_s;
+  // sequences (hence work items) of this launch: all, or the listed ones with the count read on the device
+  const int n_live = attn::live_sequences(prm);
+  const int n_items = n_live * prm.Hkv * prm.n_mtiles;
   bool timed_out = false;
 
   if (warp == kProducerWarp) {
     // ============================ TMA producer ============================
-    bool bad_index = false;
+    bool bad_index = attn::bad_sequence_numbers(prm, n_live);
     if (lane == 0) {
       auto prefetch_map = [](const CUtensorMap *m) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
@@ -238,7 +241,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       __syncwarp();
       idx_cache = cache;
     }
-    const int n_my = (prm.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // items of this CTA
+    const int n_my = (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // items of this CTA
     int q_next = 0;  // first item (in this CTA's order) whose query tile has not been requested yet
     // Requests the query tile(s) of this CTA's kq-th item.  The caller has made sure the previous
     // item's last Q K^T has completed.
@@ -361,7 +364,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     int g0 = 0;   // tiles processed by this CTA before the current item
     int k = 0;
     int gx0 = 0;  // tiles of items with extra rows before the current item
-    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
       const bool has_x = (D == 128) && decode_item(prm, item).x_rows > 0;
       ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full, k & 1, abort_flag));
       for (int j = 0; j < n_tiles && ok; ++j) {
@@ -431,7 +434,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     int g0 = 0, k = 0;
     int kx = 0;   // items with extra rows before the current one
     int gx0 = 0;  // tiles of such items
-    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
       const bool has_x = (D == 128) && decode_item(prm, item).x_rows > 0;
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int g = g0 + j, gx = gx0 + j;
@@ -508,7 +511,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       ++n_y;
       return __all_sync(0xffffffffu, w);
     };
-    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
       const Item it = decode_item(prm, item);
       if (!((D == 128) && it.x_rows > 0)) {
         // nothing to do, but stay in step with the per-item barrier (a parity wait cannot skip phases)
@@ -660,7 +663,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     (void)tracer;
     bool ok = true;
     int g0 = 0, k = 0;
-    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
       const Item it = decode_item(prm, item);
       const bool live = row < it.m_rows;
       float m_used = -INFINITY;  // maximum the probabilities are expressed against (log2 units)
@@ -822,9 +825,10 @@ int launch_d(const ds_attn_params &p, cudaStream_t stream) {
     prm.n_mtiles = n_full + (rem ? 1 : 0);
     prm.x_rows = 0;
   }
-  const long long n_items = (long long)p.B * p.Hkv * prm.n_mtiles;
+  const long long n_items = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv * prm.n_mtiles;  // upper bound with a device count
   if (n_items > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   prm.n_items = (int)n_items;
+  if (n_items == 0) return DS_OK;
   const int grid = (int)(n_items < sm_count() ? n_items : sm_count());
   attn_tc_kernel<D><<<grid, kNumThreads, Geo<D>::kSmemBytes, stream>>>(prm);
   DS_CUDA_OK(cudaGetLastError());
@@ -875,6 +879,9 @@ bool fill_common(AttnCommon &c, const ds_attn_params &p) {
   c.status = p.status;
   c.B = p.B, c.Hq = p.Hq, c.Hkv = p.Hkv, c.G = p.Hq / p.Hkv, c.P = p.P, c.T = p.T, c.Lq = p.Lq;
   c.scale_log2 = p.scale * kLog2e;
+  c.seq_list = p.seq_list;
+  c.n_seq_dev = p.seq_list ? p.n_seq_dev : nullptr;
+  c.n_seq = p.n_seq;
   return true;
 }
 }  // namespace attn

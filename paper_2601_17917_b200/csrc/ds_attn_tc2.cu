@@ -70,7 +70,7 @@ __device__ __forceinline__ Item2 decode_item2(const Tc2Params &prm, int item) {
   it.pr = item % prm.n_pairs;
   const int bh = item / prm.n_pairs;
   it.hk = bh % prm.Hkv;
-  it.b = bh / prm.Hkv;
+  it.b = listed_batch(prm, bh / prm.Hkv);
   const int left = prm.G * prm.Lq - it.pr * 2 * kBlockM;
   it.rows_a = min(kBlockM, left);
   it.rows_b = max(0, min(kBlockM, left - kBlockM));
@@ -125,11 +125,14 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_base_s;
+  // sequences (hence work items) of this launch: all, or the listed ones with the count read on the device
+  const int n_live = live_sequences(prm);
+  const int n_items = n_live * prm.Hkv * prm.n_pairs;
   bool timed_out = false;
 
   if (warp == kProducerWarp) {
     // ============================ TMA producer ============================
-    bool bad_index = false;
+    bool bad_index = bad_sequence_numbers(prm, n_live);
     if (lane == 0) {
       auto prefetch_map = [](const CUtensorMap *m) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
@@ -159,7 +162,7 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
       __syncwarp();
       idx_cache = cache;
     }
-    const int n_my = (prm.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int n_my = (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     int q_next = 0;
     auto issue_q = [&](int kq) {
       const Item2 it = decode_item2(prm, blockIdx.x + kq * gridDim.x);
@@ -292,7 +295,7 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
       }
       __syncwarp();
     };
-    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
       const bool has_b = decode_item2(prm, item).rows_b > 0;
       ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full, k & 1, abort_flag));
       for (int j = 0; j <= n_tiles && ok; ++j) {
@@ -338,7 +341,7 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
     const float c2 = prm.scale_log2;
     bool ok = true;
     int g0 = 0, k = 0;  // g0: tiles this warpgroup's M-tile has seen before the current item
-    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++k) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k) {
       const Item2 it = decode_item2(prm, item);
       const int my_rows = x ? it.rows_b : it.rows_a;
       if (my_rows == 0) {
@@ -482,9 +485,10 @@ int launch2_d(const ds_attn_params &p, cudaStream_t stream) {
   if (!fill_common(prm, p)) return DS_ERR_CUDA;
   const long long rows_total = (long long)prm.G * p.Lq;
   prm.n_pairs = (int)((rows_total + 2 * kBlockM - 1) / (2 * kBlockM));
-  const long long n_items = (long long)p.B * p.Hkv * prm.n_pairs;
+  const long long n_items = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv * prm.n_pairs;  // upper bound with a device count
   if (n_items > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   prm.n_items = (int)n_items;
+  if (n_items == 0) return DS_OK;
   const int grid = (int)(n_items < sm_count() ? n_items : sm_count());
   attn_tc2_kernel<D><<<grid, kThreads2, Geo2<D>::kSmemBytes, stream>>>(prm);
   DS_CUDA_OK(cudaGetLastError());

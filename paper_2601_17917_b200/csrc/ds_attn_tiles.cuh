@@ -24,7 +24,33 @@ struct AttnCommon {
   uint32_t *status;
   int B, Hq, Hkv, G, P, T, Lq;
   float scale_log2;  // softmax scale * log2(e)
+  // optional restriction to listed sequences (the ones whose block still has masked positions)
+  const int32_t *seq_list;   // ascending batch numbers, nullptr = all B
+  const int32_t *n_seq_dev;  // device count overriding n_seq (clamped to [0, n_seq]), may be nullptr
+  int n_seq;
 };
+
+// Number of sequences this launch processes, and the batch number of the s-th of them.
+__device__ __forceinline__ int live_sequences(const AttnCommon &c) {
+  if (c.seq_list == nullptr) return c.B;
+  int n = c.n_seq;
+  if (c.n_seq_dev != nullptr) n = max(0, min(n, *c.n_seq_dev));
+  return n;
+}
+__device__ __forceinline__ int listed_batch(const AttnCommon &c, int s) {
+  if (c.seq_list == nullptr) return s;
+  return min(max(c.seq_list[s], 0), c.B - 1);
+}
+// Producer warp: flags list entries outside [0, B) (they are clamped by listed_batch).
+__device__ __forceinline__ bool bad_sequence_numbers(const AttnCommon &c, int n_live) {
+  bool bad = false;
+  if (c.seq_list != nullptr)
+    for (int s = threadIdx.x & 31; s < n_live; s += 32) {
+      const int v = c.seq_list[s];
+      bad |= (v < 0 || v >= c.B);
+    }
+  return bad;
+}
 
 // ------------------------------------------------------------------------------------------------
 // Producer helper: fetch n gathered rows (logical rows R0 .. R0+n-1 of a stacked sequence whose

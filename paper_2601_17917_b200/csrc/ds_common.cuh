@@ -39,8 +39,8 @@ __device__ __forceinline__ float bf16hi_to_f32(uint32_t w) { return __uint_as_fl
 
 // Launchers implemented in the per-kernel translation units.
 int launch_confidence(const void *logits, int dtype, int64_t rows, int64_t V, int64_t ld,
-                      const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
-                      void *workspace, size_t workspace_bytes, cudaStream_t stream);
+                      const int32_t *row_list, int64_t n_listed, const int32_t *n_listed_dev, float *conf,
+                      int32_t *tok, void *workspace, size_t workspace_bytes, cudaStream_t stream);
 size_t confidence_workspace_bytes(int64_t rows, int64_t V, int dtype);
 int launch_confidence_static(const void *logits, int dtype, int64_t rows, int64_t V, int64_t ld,
                              const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,

@@ -139,11 +139,13 @@ __global__ void __launch_bounds__(kThreads)
 confidence_kernel(const T *__restrict__ logits, long long V, long long ld,
                   const int32_t *__restrict__ row_list, int splits, float *__restrict__ conf,
                   int32_t *__restrict__ tok, Triple *__restrict__ partials,
-                  unsigned *__restrict__ tickets) {
+                  unsigned *__restrict__ tickets, const int32_t *__restrict__ n_listed_dev, long long rows) {
   constexpr int N = Vec<T>::N;
   const int li = blockIdx.x / splits;  // position in the list of processed rows
   const int sp = blockIdx.x - li * splits;
+  if (n_listed_dev != nullptr && li >= *n_listed_dev) return;  // the list is shorter than the launch was sized for
   const long long row = row_list ? (long long)row_list[li] : (long long)li;
+  if (row < 0 || row >= rows) return;  // every CTA of the row leaves: no ticket of it is ever awaited
   const T *z = logits + row * ld;
   const int tid = threadIdx.x;
 
@@ -290,6 +292,7 @@ int static_scratch(void **out) {
 int launch_confidence_static(const void *logits, int dtype, int64_t rows, int64_t V, int64_t ld,
                              const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
                              cudaStream_t stream) {
+  const int32_t *n_listed_dev = nullptr;
   const int64_t n = row_list ? n_listed : rows;
   if (n == 0) return DS_OK;
   if (n > kStaticRows) return DS_ERR_STATIC_LIMIT;
@@ -305,10 +308,10 @@ int launch_confidence_static(const void *logits, int dtype, int64_t rows, int64_
   const dim3 grid((unsigned)(n * splits));
   if (dtype == DS_BF16) {
     confidence_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>(
-        reinterpret_cast<const __nv_bfloat16 *>(logits), V, ld, row_list, splits, conf, tok, partials, tickets);
+        reinterpret_cast<const __nv_bfloat16 *>(logits), V, ld, row_list, splits, conf, tok, partials, tickets, n_listed_dev, rows);
   } else {
     confidence_kernel<float><<<grid, kThreads, 0, stream>>>(reinterpret_cast<const float *>(logits), V, ld,
-                                                           row_list, splits, conf, tok, partials, tickets);
+                                                           row_list, splits, conf, tok, partials, tickets, n_listed_dev, rows);
   }
   DS_CUDA_OK(cudaGetLastError());
   note_launch(1);
@@ -323,8 +326,8 @@ size_t confidence_workspace_bytes(int64_t rows, int64_t V, int dtype) {
 }
 
 int launch_confidence(const void *logits, int dtype, int64_t rows, int64_t V, int64_t ld,
-                      const int32_t *row_list, int64_t n_listed, float *conf, int32_t *tok,
-                      void *workspace, size_t workspace_bytes, cudaStream_t stream) {
+                      const int32_t *row_list, int64_t n_listed, const int32_t *n_listed_dev, float *conf,
+                      int32_t *tok, void *workspace, size_t workspace_bytes, cudaStream_t stream) {
   const int64_t n = row_list ? n_listed : rows;
   if (n == 0) return DS_OK;
   const int splits = pick_splits(n, V, dtype);
@@ -343,10 +346,10 @@ int launch_confidence(const void *logits, int dtype, int64_t rows, int64_t V, in
   const dim3 grid((unsigned)(n * splits));
   if (dtype == DS_BF16) {
     confidence_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>(
-        reinterpret_cast<const __nv_bfloat16 *>(logits), V, ld, row_list, splits, conf, tok, partials, tickets);
+        reinterpret_cast<const __nv_bfloat16 *>(logits), V, ld, row_list, splits, conf, tok, partials, tickets, n_listed_dev, rows);
   } else {
     confidence_kernel<float><<<grid, kThreads, 0, stream>>>(reinterpret_cast<const float *>(logits), V, ld,
-                                                           row_list, splits, conf, tok, partials, tickets);
+                                                           row_list, splits, conf, tok, partials, tickets, n_listed_dev, rows);
   }
   DS_CUDA_OK(cudaGetLastError());
   note_launch(1);

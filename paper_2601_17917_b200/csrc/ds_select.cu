@@ -140,6 +140,54 @@ __device__ void compact_active(const ds_select_params &p, int n) {
   if (tid == 0) *p.active_cnt = running;
 }
 
+// Ordered list of the rows b * K + i that are still masked, over the processed sequences in list order.
+// Runs in one CTA of kSelThreads threads after the selection: one sequence per warp, kSelWarps per round.
+__device__ void compact_masked_rows(const ds_select_params &p, int n) {
+  __shared__ int rem_cnt[kSelWarps];
+  __shared__ int rows_so_far;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int K = p.K;
+  if (tid == 0) rows_so_far = 0;
+  __syncthreads();
+  for (int s0 = 0; s0 < n; s0 += kSelWarps) {
+    const int s = s0 + wid;
+    int b = -1;
+    if (s < n) {
+      b = p.seq_list ? p.seq_list[s] : s;
+      if (b < 0 || b >= p.B) b = -1;
+    }
+    const uint8_t *mk = p.masked + (long long)(b < 0 ? 0 : b) * K;
+    int rem = 0;
+    if (b >= 0) {
+      for (int base = 0; base < K; base += 32) {
+        const int i = base + lane;
+        rem += __popc(__ballot_sync(0xffffffffu, (i < K) && (mk[i] != 0)));
+      }
+    }
+    if (lane == 0) rem_cnt[wid] = rem;
+    __syncthreads();
+    int off = rows_so_far;
+    for (int w = 0; w < wid; ++w) off += rem_cnt[w];
+    if (b >= 0 && rem > 0) {
+      for (int base = 0; base < K; base += 32) {
+        const int i = base + lane;
+        const bool m = (i < K) && (mk[i] != 0);
+        const unsigned bal = __ballot_sync(0xffffffffu, m);
+        if (m) p.masked_rows[off + __popc(bal & ((1u << lane) - 1u))] = b * K + i;
+        off += __popc(bal);
+      }
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int tot = 0;
+      for (int w = 0; w < kSelWarps; ++w) tot += rem_cnt[w];
+      rows_so_far += tot;
+    }
+    __syncthreads();
+  }
+  if (tid == 0) *p.masked_cnt = rows_so_far;
+}
+
 __global__ void __launch_bounds__(kSelThreads) select_fused_kernel(const ds_select_params p) {
   const int n = listed_count(p);
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -147,8 +195,9 @@ __global__ void __launch_bounds__(kSelThreads) select_fused_kernel(const ds_sele
     const int b = p.seq_list ? p.seq_list[s] : s;
     if (b >= 0 && b < p.B) select_sequence(p, b, lane);
   }
-  __syncthreads();  // block_done of every sequence written by this CTA is visible below
+  __syncthreads();  // block_done and the mask flags of every sequence written by this CTA are visible below
   compact_active(p, n);
+  if (p.masked_rows != nullptr) compact_masked_rows(p, n);
 }
 
 __global__ void __launch_bounds__(256) select_grid_kernel(const ds_select_params p) {
@@ -161,7 +210,9 @@ __global__ void __launch_bounds__(256) select_grid_kernel(const ds_select_params
 }
 
 __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const ds_select_params p) {
-  compact_active(p, listed_count(p));
+  const int n = listed_count(p);
+  compact_active(p, n);
+  if (p.masked_rows != nullptr) compact_masked_rows(p, n);
 }
 
 }  // namespace

@@ -262,3 +262,40 @@ def test_full_size_unpruned_reference_sampled_rows():
 def test_cache_refresh_step_dense_no_prefix():
     # first step of a block: no cached prefix, every row of the sequence is a query and a key (Lq = Lkv = 2048)
     _sampled_parity(wl.CONFIGS["refresh8"], n_slices=4, q_rows=16)
+
+
+@pytest.mark.parametrize("path,dtype,Lq", [("simt", torch.float32, 40), ("tc", torch.bfloat16, 97),
+                                           ("tc", torch.bfloat16, 300), ("tc2", torch.bfloat16, 300)])
+def test_listed_sequences_only(path, dtype, Lq, monkeypatch):
+    # a step restricted to the sequences whose block is unfinished: list and count on the device
+    monkeypatch.setenv("DS_ATTN_PATH", path)
+    B, Hq, Hkv, D, P, T = 5, 4, 2, 128, 200, 320
+    g = torch.Generator().manual_seed(77)
+    mk = lambda *sh: torch.randn(*sh, generator=g).to(dtype).to(DEV)
+    q, kt, vt, kp, vp = mk(B, Hq, T, D), mk(B, Hkv, T, D), mk(B, Hkv, T, D), mk(B, Hkv, P, D), mk(B, Hkv, P, D)
+    idx = np.arange(Lq, dtype=np.int32)
+    idx[Lq - 1] = T - 1
+    idx_t = torch.tensor(idx, device=DEV)
+    scale = 1.0 / math.sqrt(D)
+    ref = oracle.attn(_np(q), _np(kt), _np(vt), _np(kp), _np(vp), idx, scale)
+    lst = torch.tensor([1, 3, 4, 0, 0], dtype=torch.int32, device=DEV)   # entries past the count are ignored
+    for n_dev, n_host in ((3, 5), (2, 5), (0, 5), (None, 2)):
+        out = torch.full((B, Hq, Lq, D), 123.0, dtype=dtype, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        cnt = None if n_dev is None else torch.tensor([n_dev], dtype=torch.int32, device=DEV)
+        ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, out=out, status=status, seq_list=lst, n_seq=n_host,
+                          n_seq_dev=cnt)
+        torch.cuda.synchronize()
+        assert ds.ds_read_status(status) == 0
+        live = lst[: (n_host if n_dev is None else n_dev)].cpu().tolist()
+        for b in range(B):
+            if b in live:
+                _compare(out[b], ref[b], dtype, f"{path} seq {b}")
+            else:
+                assert (out[b] == 123.0).all(), f"sequence {b} is not listed and must stay untouched"
+    # a sequence number outside [0, B) is reported
+    bad = torch.tensor([1, 9], dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, status=status, seq_list=bad)
+    torch.cuda.synchronize()
+    assert ds.ds_read_status(status) & ds.DS_DEV_INDEX

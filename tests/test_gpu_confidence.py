@@ -22,7 +22,7 @@ def _check(z_dev, conf, tok, rows=None):
     z = z_dev.float().cpu().numpy()
     rc, rt = oracle.confidence(z)
     conf, tok = conf.cpu().numpy(), tok.cpu().numpy()
-    sel = np.arange(z.shape[0]) if rows is None else np.asarray(rows)
+    sel = np.arange(z.shape[0]) if rows is None else np.asarray(rows, dtype=np.int64)
     assert (tok[sel] == rt[sel]).all(), "argmax mismatch"
     err = np.abs(conf[sel].astype(np.float64) - rc[sel]).max() if len(sel) else 0.0
     assert err <= CONF_BAR and err <= CONF_OWN, err
@@ -125,3 +125,30 @@ def test_workspace_errors_and_determinism():
         if first is None:
             first = cur
         assert torch.equal(cur[0], first[0]) and torch.equal(cur[1], first[1])   # bitwise repeatable
+
+
+@pytest.mark.parametrize("V", [1000, 126464])
+def test_listed_rows_with_the_count_on_the_device(V):
+    # the rows still masked and their number live on the device (ds_unmask_select's masked_rows / masked_cnt)
+    torch.manual_seed(5)
+    rows = 96
+    z = (torch.randn(rows, V, device=DEV) * 3).to(torch.bfloat16)
+    lst = torch.tensor([3, 4, 17, 40, 41, 42, 90, 95, 1, 2], dtype=torch.int32, device=DEV)  # the last two: beyond the count
+    for n in (8, 0, 3):
+        conf = torch.full((rows,), -7.0, device=DEV)
+        tok = torch.full((rows,), -7, dtype=torch.int32, device=DEV)
+        cnt = torch.tensor([n], dtype=torch.int32, device=DEV)
+        ds.ds_confidence_listed(z, lst, cnt, conf, tok)
+        torch.cuda.synchronize()
+        used = lst[:n].cpu().tolist()
+        _check(z, conf, tok, rows=used)
+        rest = sorted(set(range(rows)) - set(used))
+        assert (conf[rest] == -7.0).all() and (tok[rest] == -7).all()
+    # a count larger than the list is clamped to the list; a row number outside the matrix is skipped
+    lst2 = torch.tensor([5, 6, 1000, -1], dtype=torch.int32, device=DEV)
+    conf = torch.full((rows,), -7.0, device=DEV)
+    tok = torch.full((rows,), -7, dtype=torch.int32, device=DEV)
+    ds.ds_confidence_listed(z, lst2, torch.tensor([99], dtype=torch.int32, device=DEV), conf, tok)
+    torch.cuda.synchronize()
+    _check(z, conf, tok, rows=[5, 6])
+    assert (conf[7:] == -7.0).all()

@@ -34,22 +34,31 @@ def _gpu_select(conf, tok, masked, x, **kw):
                eos_exit=(torch.zeros(B, dtype=torch.uint8, device=DEV) if eos_init is None
                          else torch.as_tensor(eos_init, dtype=torch.uint8).to(DEV)),
                active_seq=torch.full((max(B, 1),), -5, dtype=torch.int32, device=DEV),
-               active_cnt=torch.full((1,), -5, dtype=torch.int32, device=DEV))
+               active_cnt=torch.full((1,), -5, dtype=torch.int32, device=DEV),
+               masked_rows=torch.full((max(B * K, 1),), -5, dtype=torch.int32, device=DEV),
+               masked_cnt=torch.full((1,), -5, dtype=torch.int32, device=DEV))
     ds.ds_unmask_select(c, t, m, xb, out=out, **kw)
     torch.cuda.synchronize()
     n = int(out["active_cnt"].item())
-    return dict(masked=m.cpu().numpy(), x_block=xb.cpu().numpy(), sel_idx=out["sel_idx"].cpu().numpy(),
+    nr = int(out["masked_cnt"].item())
+    assert (out["masked_rows"][nr:] == -5).all()
+    return dict(masked_rows=out["masked_rows"].cpu().numpy()[:nr], masked=m.cpu().numpy(), x_block=xb.cpu().numpy(), sel_idx=out["sel_idx"].cpu().numpy(),
                 sel_cnt=out["sel_cnt"].cpu().numpy(), block_done=out["block_done"].cpu().numpy(),
                 eos_exit=out["eos_exit"].cpu().numpy(), active_seq=out["active_seq"].cpu().numpy()[:n])
 
 
 def _same(g, o, seqs=None):
     B = g["masked"].shape[0]
-    seqs = range(B) if seqs is None else seqs
+    seqs = list(range(B)) if seqs is None else list(seqs)
     for b in seqs:
         for k in ("masked", "x_block", "sel_idx", "sel_cnt", "block_done", "eos_exit"):
             assert np.array_equal(g[k][b], o[k][b]), (k, b, g[k][b], o[k][b])
     assert g["active_seq"].tolist() == o["active_seq"].tolist()
+    # the rows still masked after the step, over the processed sequences (all of them when none are listed)
+    if seqs is not None:
+        K = o["masked"].shape[1]
+        want = [b * K + i for b in sorted(seqs) for i in np.nonzero(o["masked"][b])[0]]
+        assert g["masked_rows"].tolist() == want
 
 
 @pytest.mark.parametrize("name", ["tiny", "llada1", "llada8x32", "dream16", "long32-w64"])
