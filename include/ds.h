@@ -323,6 +323,38 @@ typedef struct {
 DS_API int ds_unmask_select(const ds_select_params *p, void *stream);
 
 /* ------------------------------------------------------------------------
+ * ds_block_begin  (Eq. 1, Eq. 2, block termination rule, early exit)
+ *
+ * Decoding proceeds block by block: when block n has no masked position left
+ * "the model proceeds to decode block n+1", and once a sequence has predicted
+ * EOS with high confidence "all subsequent blocks are skipped".  This entry
+ * point prepares the device state of the next block from the per-sequence
+ * early-exit flags, without the host looking at them:
+ *     for b with eos_exit[b] == 0:  masked[b][:] = 1, x_block[b][:] = mask_id   (Eq. 1: K fresh [MASK])
+ *     for b with eos_exit[b] != 0:  masked[b][:] = 0, x_block[b][:] = fill_id   (block skipped)
+ *     active_seq  = ascending list of the b with eos_exit[b] == 0, *active_cnt its length
+ *     masked_rows = b * K + i for those b (list order) and i = 0..K-1, *masked_cnt = *active_cnt * K
+ * in the layout ds_unmask_select, ds_confidence_listed and ds_attn_pruned's
+ * seq_list read.  masked_rows/masked_cnt are optional (both NULL or both set).
+ * Errors: DS_ERR_INVALID_ARG (NULL pointer, B < 0, K outside 1..4096), DS_ERR_UNSUPPORTED (B * K > 2^31 - 1).
+ * ------------------------------------------------------------------------ */
+typedef struct {
+  int32_t B, K;
+  int32_t mask_id;              /* token id of [MASK] */
+  int32_t fill_id;              /* token written to the block of a sequence that has exited (normally EOS) */
+  const uint8_t *eos_exit;      /* [B] */
+  uint8_t *masked;              /* [B][K] out */
+  int32_t *x_block;             /* [B][K] out */
+  int32_t *active_seq;          /* [B] out */
+  int32_t *active_cnt;          /* [1] out */
+  int32_t *masked_rows;         /* optional [B*K] out */
+  int32_t *masked_cnt;          /* optional [1] out */
+} ds_block_params;
+
+/* `p` is a HOST pointer; the pointers inside it are device pointers. */
+DS_API int ds_block_begin(const ds_block_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
  * Utilities
  * ------------------------------------------------------------------------ */
 /* Copies the device status word to *host_out (HOST) after synchronising `stream`. */

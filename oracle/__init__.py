@@ -22,6 +22,10 @@ Contents
   logits) composed with Eq. 4, logits kept in float64.
 * ``threshold`` / ``select`` (C, float32, contraction off): Eq. 10, Eq. 9, Eq. 5,
   block termination and the early-exit flag.
+* ``decode`` (Python loop over the above): the block-wise decoding procedure of
+  the Preliminary section (Eq. 1-5) with the selection rule of Eq. 9-10 and
+  "Early Exit For Block Diffusion", the model being a caller-supplied function
+  that returns the current block's logits.
 
 Pins (see tests, run with ``-m "not gpu"``): every function is checked against
 closed forms, invariants, a library routine on the special case it reduces to,
@@ -282,3 +286,60 @@ def select(conf, tok, masked, x_block, tau0, alpha, ratio_extra=0, eos_id=-1, eo
         raise ValueError("oracle_select rejected its arguments")
     return dict(masked=masked, x_block=x_block, sel_idx=sel_idx, sel_cnt=sel_cnt, block_done=block_done,
                 eos_exit=eos, active_seq=active[: int(n_active[0])].copy(), tau=tau)
+
+
+# --------------------------------------------------------------------------
+# the block-wise decoding procedure
+# --------------------------------------------------------------------------
+def decode(logits_fn, B: int, L: int, K: int, tau0: float, alpha: float, mask_id: int, eos_id: int = -1,
+           eos_tau: float = 0.9, extra_fn=None, trace=None):
+    """Block-wise diffusion decoding of B sequences (Preliminary, Eq. 1-5; selection by Eq. 9-10;
+    "Early Exit For Block Diffusion").
+
+    Eq. 1: the generated part starts as L [MASK] tokens, split (Eq. 2) into N = L / K blocks.  Block n is
+    iterated until none of its positions is masked, then block n + 1 follows.  At iteration t of block n
+    ``logits_fn(n, t)`` stands for Eq. 3 and returns the logits [B, K, V] of the block's positions;
+    Eq. 4 gives confidences and tokens, Eq. 9-10 choose the positions to finalise, Eq. 5 updates them.
+    Sequences whose block is finished are no longer processed (their logits are not looked at).
+    Early exit: a sequence that finalised ``eos_id`` with confidence >= ``eos_tau`` finishes its current
+    block and skips every later block; the skipped blocks are filled with ``eos_id`` (the paper only says
+    the sequence "remains complete").
+    ``extra_fn(n)`` = number of retained suffix rows counted as masked in Eq. 10's ratio (None: 0).
+
+    Returns dict(x [B, L] int32, steps [N] iterations spent on each block, seq_steps [B, N] iterations
+    each sequence took part in, eos_exit [B]).  ``trace``, if a list, receives one dict per iteration
+    (n, t, conf, tau, masked before, active before).
+    """
+    if L % K != 0:
+        raise ValueError("L must be a multiple of K")
+    N = L // K
+    x = np.full((B, L), mask_id, dtype=np.int32)
+    steps = np.zeros(N, dtype=np.int32)
+    seq_steps = np.zeros((B, N), dtype=np.int32)
+    exited = np.zeros(B, dtype=np.uint8)
+    for n in range(N):
+        live = [b for b in range(B) if exited[b] == 0]
+        masked = np.zeros((B, K), dtype=np.uint8)
+        xb = np.full((B, K), eos_id, dtype=np.int32)
+        masked[live] = 1
+        xb[live] = mask_id
+        extra = 0 if extra_fn is None else int(extra_fn(n))
+        active = list(live)
+        t = 0
+        while active:
+            z = np.asarray(logits_fn(n, t), dtype=np.float64)
+            V = z.shape[-1]
+            conf, tok = confidence(z.reshape(B * K, V))
+            conf = conf.reshape(B, K).astype(np.float32)   # Eq. 9's comparison is taken in float32
+            tok = tok.reshape(B, K)
+            r = select(conf, tok, masked, xb, tau0, alpha, ratio_extra=extra, eos_id=eos_id, eos_tau=eos_tau,
+                       seq_list=active, eos_exit=exited)
+            if trace is not None:
+                trace.append(dict(n=n, t=t, conf=conf, tau=r["tau"], masked=masked.copy(), active=list(active)))
+            seq_steps[active, n] += 1
+            masked, xb, exited = r["masked"], r["x_block"], r["eos_exit"]
+            active = r["active_seq"].tolist()
+            t += 1
+        steps[n] = t
+        x[:, n * K:(n + 1) * K] = xb
+    return dict(x=x, steps=steps, seq_steps=seq_steps, eos_exit=exited)

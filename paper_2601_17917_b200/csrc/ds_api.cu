@@ -209,6 +209,15 @@ int ds_unmask_select(const ds_select_params *p, void *stream) {
   return ds::launch_select(*p, reinterpret_cast<cudaStream_t>(stream));
 }
 
+int ds_block_begin(const ds_block_params *p, void *stream) {
+  if (!p) return DS_ERR_INVALID_ARG;
+  if (p->B < 0 || p->K < 1 || p->K > 4096) return DS_ERR_INVALID_ARG;
+  if (!p->active_cnt || (p->masked_rows == nullptr) != (p->masked_cnt == nullptr)) return DS_ERR_INVALID_ARG;
+  if ((long long)p->B * p->K > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
+  if (p->B > 0 && (!p->eos_exit || !p->masked || !p->x_block || !p->active_seq)) return DS_ERR_INVALID_ARG;
+  return ds::launch_block_begin(*p, reinterpret_cast<cudaStream_t>(stream));
+}
+
 int ds_read_status(const uint32_t *device_status, void *stream, uint32_t *host_out) {
   if (!device_status || !host_out) return DS_ERR_INVALID_ARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);

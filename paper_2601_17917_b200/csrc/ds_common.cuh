@@ -49,6 +49,7 @@ size_t lmhead_workspace_bytes(int64_t rows, int64_t V);
 int launch_lmhead_confidence(const void *hidden, const void *weight, int64_t rows, int64_t hid, int64_t V, int64_t ld_h,
                              int64_t ld_w, float *conf, int32_t *tok, void *workspace, uint32_t *status,
                              cudaStream_t stream);
+int launch_block_begin(const ds_block_params &p, cudaStream_t stream);
 int launch_select(const ds_select_params &p, cudaStream_t stream);
 int launch_rope_gather(const ds_rope_params &p, cudaStream_t stream);
 int launch_attn_simt(const ds_attn_params &p, cudaStream_t stream);

@@ -215,7 +215,60 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const ds_se
   if (p.masked_rows != nullptr) compact_masked_rows(p, n);
 }
 
+// Start of a block: mask flags, block tokens and the lists of the sequences that have not exited.
+__global__ void __launch_bounds__(kSelThreads) block_begin_kernel(const ds_block_params p) {
+  __shared__ int warp_cnt[kSelWarps];
+  __shared__ int running;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) running = 0;
+  __syncthreads();
+  for (int base = 0; base < p.B; base += kSelThreads) {  // ordered compaction of the live sequences
+    const int b = base + tid;
+    const bool live = (b < p.B) && (p.eos_exit[b] == 0);
+    const unsigned bal = __ballot_sync(0xffffffffu, live);
+    if (lane == 0) warp_cnt[wid] = __popc(bal);
+    __syncthreads();
+    int off = running;
+    for (int w = 0; w < wid; ++w) off += warp_cnt[w];
+    if (live) p.active_seq[off + __popc(bal & ((1u << lane) - 1u))] = b;
+    __syncthreads();
+    if (tid == 0) {
+      int tot = 0;
+      for (int w = 0; w < kSelWarps; ++w) tot += warp_cnt[w];
+      running += tot;
+    }
+    __syncthreads();
+  }
+  const int n_live = running;
+  if (tid == 0) {
+    *p.active_cnt = n_live;
+    if (p.masked_cnt) *p.masked_cnt = n_live * p.K;
+  }
+  // one warp per sequence: its K flags and tokens
+  for (int b = wid; b < p.B; b += kSelWarps) {
+    const bool live = p.eos_exit[b] == 0;
+    for (int i = lane; i < p.K; i += 32) {
+      p.masked[(long long)b * p.K + i] = live ? 1 : 0;
+      p.x_block[(long long)b * p.K + i] = live ? p.mask_id : p.fill_id;
+    }
+  }
+  if (p.masked_rows) {
+    __syncthreads();  // active_seq as written above by this CTA
+    for (int a = wid; a < n_live; a += kSelWarps) {
+      const int b = p.active_seq[a];
+      for (int i = lane; i < p.K; i += 32) p.masked_rows[(long long)a * p.K + i] = b * p.K + i;
+    }
+  }
+}
+
 }  // namespace
+
+int launch_block_begin(const ds_block_params &p, cudaStream_t stream) {
+  block_begin_kernel<<<1, kSelThreads, 0, stream>>>(p);
+  DS_CUDA_OK(cudaGetLastError());
+  note_launch(1);
+  return DS_OK;
+}
 
 int launch_select(const ds_select_params &p, cudaStream_t stream) {
   const int n = p.seq_list ? p.n_seq : p.B;
