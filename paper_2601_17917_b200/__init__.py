@@ -20,7 +20,7 @@ __all__ = [
     "lib", "retained_indices", "ds_attn_pruned", "ds_attn_pruned_workspace", "ds_confidence",
     "ds_confidence_workspace", "ds_confidence_static", "ds_lmhead_confidence", "ds_lmhead_confidence_workspace",
     "ds_rope_gather", "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
-    "ds_launch_count", "DsError", "DS_F32", "DS_BF16", "DS_DEV_INDEX", "DS_DEV_TIMEOUT",
+    "ds_launch_count", "ds_block_begin", "ds_confidence_listed", "DsError", "DS_F32", "DS_BF16", "DS_DEV_INDEX", "DS_DEV_TIMEOUT",
 ]
 
 DS_F32, DS_BF16 = 0, 1
@@ -65,6 +65,15 @@ class _RopeParams(ctypes.Structure):
         ("q_out_stride", ctypes.c_int64 * 3), ("kv_out_stride", ctypes.c_int64 * 3),
         ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p), ("cache_stride", ctypes.c_int64 * 3),
         ("cache_row0", ctypes.c_int32), ("n_append", ctypes.c_int32), ("status", ctypes.c_void_p),
+    ]
+
+
+class _BlockParams(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("K", ctypes.c_int32), ("mask_id", ctypes.c_int32), ("fill_id", ctypes.c_int32),
+        ("eos_exit", ctypes.c_void_p), ("masked", ctypes.c_void_p), ("x_block", ctypes.c_void_p),
+        ("active_seq", ctypes.c_void_p), ("active_cnt", ctypes.c_void_p), ("masked_rows", ctypes.c_void_p),
+        ("masked_cnt", ctypes.c_void_p),
     ]
 
 
@@ -114,6 +123,8 @@ def lib() -> ctypes.CDLL:
         L.ds_confidence_static.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                            ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                            ctypes.c_void_p, ctypes.c_void_p]
+        L.ds_block_begin.restype = ctypes.c_int
+        L.ds_block_begin.argtypes = [ctypes.POINTER(_BlockParams), ctypes.c_void_p]
         L.ds_unmask_select.restype = ctypes.c_int
         L.ds_unmask_select.argtypes = [ctypes.POINTER(_SelectParams), ctypes.c_void_p]
         L.ds_read_status.restype = ctypes.c_int
@@ -444,6 +455,30 @@ def ds_unmask_select(conf, tok, masked, x_block, tau0, alpha, ratio_extra=0, eos
     if rc != DS_OK:
         raise DsError(rc, "ds_unmask_select")
     return out
+
+
+def ds_block_begin(eos_exit, masked, x_block, mask_id, fill_id, active_seq, active_cnt, masked_rows=None,
+                   masked_cnt=None, stream=None):
+    """Start of a block (Eq. 1-2, early exit): fresh [MASK] state for the sequences that have not exited,
+    ``fill_id`` for the others, and the device lists the step's entry points read."""
+    _check_dev(eos_exit, masked, x_block, active_seq, active_cnt, masked_rows, masked_cnt)
+    B, K = masked.shape
+    if eos_exit.dtype != torch.uint8 or masked.dtype != torch.uint8 or x_block.dtype != torch.int32:
+        raise TypeError("eos_exit/masked must be uint8 and x_block int32")
+    if not (masked.is_contiguous() and x_block.is_contiguous()) or tuple(x_block.shape) != (B, K):
+        raise ValueError("masked and x_block must be contiguous [B,K]")
+    for t in (active_seq, active_cnt, masked_rows, masked_cnt):
+        if t is not None and t.dtype != torch.int32:
+            raise TypeError("the lists and counts must be int32")
+    p = _BlockParams()
+    p.B, p.K, p.mask_id, p.fill_id = B, K, int(mask_id), int(fill_id)
+    p.eos_exit, p.masked, p.x_block = eos_exit.data_ptr(), masked.data_ptr(), x_block.data_ptr()
+    p.active_seq, p.active_cnt = active_seq.data_ptr(), active_cnt.data_ptr()
+    p.masked_rows = masked_rows.data_ptr() if masked_rows is not None else None
+    p.masked_cnt = masked_cnt.data_ptr() if masked_cnt is not None else None
+    rc = lib().ds_block_begin(ctypes.byref(p), _stream(stream))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_block_begin")
 
 
 def ds_read_status(status: torch.Tensor, stream=None) -> int:

@@ -1,0 +1,123 @@
+"""Block scheduler of the decoding procedure (Preliminary Eq. 1-5, the selection rule Eq. 9-10 and
+"Early Exit For Block Diffusion"): blocks in order, iterations of a block until none of its positions is
+masked, later blocks skipped for sequences that predicted EOS with high confidence.
+
+Everything the procedure decides lives on the device: which sequences still take part (``active_seq`` /
+``active_cnt``), which logit rows still need Eq. 4 (``masked_rows`` / ``masked_cnt``), the early-exit flags.
+The kernels of an iteration read those lists themselves, so the host can enqueue iterations without waiting
+for the previous one; it only looks, ``lookahead`` iterations late and through pinned memory, at the number
+of active sequences to know when to stop enqueueing iterations of a block.  ``lookahead = 0`` is the
+synchronous loop (one host wait per iteration, no surplus launch); with ``lookahead = n`` at most n surplus
+iterations per block are enqueued, and they find empty lists and do nothing.
+
+The model itself (Eq. 3) is the caller's: ``forward(step)`` must leave the logits of the current block's
+positions in ``step.logits`` using ``step.idx`` (retained rows, Eq. 7), ``step.refresh`` (first iteration of
+a block: every position is a query and the prefix cache is rebuilt) and the device lists.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import torch
+
+from . import (ds_block_begin, ds_confidence_listed, ds_confidence_workspace, ds_unmask_select,
+               retained_indices)
+
+
+@dataclass
+class Step:
+    """What ``forward`` gets for one iteration.  All tensors are device tensors owned by the decoder."""
+    n: int                      # block number
+    t: int                      # iteration within the block
+    refresh: bool               # first iteration of the block: full forward, rebuilds the prefix KV cache
+    idx: torch.Tensor           # int32 tail-relative retained rows (Eq. 7); on refresh: every row of the tail
+    active_seq: torch.Tensor    # int32 [B] sequences whose block still has masked positions (first *active_cnt)
+    active_cnt: torch.Tensor    # int32 [1]
+    x_block: torch.Tensor       # int32 [B, K] current tokens of the block ([MASK] where undecided)
+    logits: torch.Tensor        # [B * K, V] to be filled for the rows of the active sequences
+
+
+class BlockDecoder:
+    def __init__(self, B: int, L: int, K: int, V: int, *, tau0: float, alpha: float, mask_id: int, eos_id: int = -1,
+                 eos_tau: float = 0.9, w_tokens: int = 0, keep_last: bool = True, count_suffix: bool = False,
+                 logits_dtype=torch.bfloat16, device="cuda:0", lookahead: int = 2):
+        if L % K != 0:
+            raise ValueError("the generation length must be a multiple of the block size (Eq. 2)")
+        if lookahead < 0:
+            raise ValueError("lookahead must be >= 0")
+        dev = torch.device(device)
+        self.B, self.L, self.K, self.V, self.N = B, L, K, V, L // K
+        self.tau0, self.alpha, self.mask_id, self.eos_id, self.eos_tau = tau0, alpha, mask_id, eos_id, eos_tau
+        self.count_suffix, self.lookahead, self.device = count_suffix, lookahead, dev
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.x = torch.empty((B, L), **i32)
+        self.masked = torch.empty((B, K), dtype=torch.uint8, device=dev)
+        self.x_block = torch.empty((B, K), **i32)
+        self.conf = torch.zeros(B * K, dtype=torch.float32, device=dev)
+        self.tok = torch.zeros(B * K, **i32)
+        self.logits = torch.zeros((B * K, V), dtype=logits_dtype, device=dev)
+        self.eos_exit = torch.zeros(B, dtype=torch.uint8, device=dev)
+        # the active list is read and rewritten by the same selection kernel: two copies, used alternately
+        self.active = [torch.zeros(max(B, 1), **i32) for _ in range(2)]
+        self.active_cnt = [torch.zeros(1, **i32) for _ in range(2)]
+        self.sel = [dict(sel_idx=torch.empty((B, K), **i32), sel_cnt=torch.zeros(B, **i32),
+                         block_done=torch.zeros(B, dtype=torch.uint8, device=dev), eos_exit=self.eos_exit,
+                         active_seq=self.active[k], active_cnt=self.active_cnt[k],
+                         masked_rows=None, masked_cnt=None) for k in range(2)]
+        self.masked_rows = torch.zeros(max(B * K, 1), **i32)
+        self.masked_cnt = torch.zeros(1, **i32)
+        for s in self.sel:
+            s["masked_rows"], s["masked_cnt"] = self.masked_rows, self.masked_cnt
+        self.workspace = torch.empty(max(ds_confidence_workspace(B * K, V, logits_dtype), 1), dtype=torch.uint8,
+                                     device=dev)
+        # Eq. 7 per block: the retained rows of the pruned iterations and all rows for the refresh iteration
+        self.idx, self.idx_all, self.extra = [], [], []
+        for n in range(self.N):
+            keep = retained_indices(L, K, n, w_tokens, keep_last)
+            self.idx.append(torch.tensor(keep, **i32))
+            self.idx_all.append(torch.arange(L - n * K, **i32))
+            self.extra.append(len(keep) - K if count_suffix else 0)
+        # slot j of a block: number of active sequences before iteration j, copied to pinned memory
+        self.cnt_host = torch.zeros(K + 1, dtype=torch.int32).pin_memory()
+        self.events = [torch.cuda.Event() for _ in range(K + 1)]
+
+    def _publish(self, slot: int, cnt: torch.Tensor):
+        self.cnt_host[slot:slot + 1].copy_(cnt, non_blocking=True)
+        self.events[slot].record()
+
+    def decode(self, forward) -> dict:
+        """Runs the whole procedure on the current stream.  Returns x [B, L] (device), steps [N] (iterations
+        each block needed), launched [N] (iterations enqueued, >= steps) and eos_exit [B] (device)."""
+        B, K, N = self.B, self.K, self.N
+        self.x.fill_(self.mask_id)
+        self.eos_exit.zero_()
+        steps, launched = [], []
+        for n in range(N):
+            ds_block_begin(self.eos_exit, self.masked, self.x_block, self.mask_id, self.eos_id, self.active[0],
+                           self.active_cnt[0], self.masked_rows, self.masked_cnt)
+            self._publish(0, self.active_cnt[0])
+            cur, t = 0, 0
+            while t < K:
+                seen = t - self.lookahead            # the newest slot the host insists on having seen
+                if seen >= 0:
+                    self.events[seen].synchronize()
+                    if int(self.cnt_host[seen]) == 0:
+                        break
+                forward(Step(n=n, t=t, refresh=(t == 0), idx=self.idx_all[n] if t == 0 else self.idx[n],
+                             active_seq=self.active[cur], active_cnt=self.active_cnt[cur], x_block=self.x_block,
+                             logits=self.logits))
+                ds_confidence_listed(self.logits, self.masked_rows, self.masked_cnt, self.conf, self.tok,
+                                     n_listed_max=B * K, workspace=self.workspace)
+                ds_unmask_select(self.conf.view(B, K), self.tok.view(B, K), self.masked, self.x_block, self.tau0,
+                                 self.alpha, ratio_extra=self.extra[n], eos_id=self.eos_id, eos_tau=self.eos_tau,
+                                 seq_list=self.active[cur], n_seq=B, n_seq_dev=self.active_cnt[cur],
+                                 out=self.sel[cur ^ 1])
+                cur ^= 1
+                t += 1
+                self._publish(t, self.active_cnt[cur])
+            self.events[t].synchronize()             # everything enqueued for this block has run
+            need = next(j for j in range(t + 1) if int(self.cnt_host[j]) == 0)
+            steps.append(need)
+            launched.append(t)
+            self.x[:, n * K:(n + 1) * K].copy_(self.x_block)
+        return dict(x=self.x, steps=steps, launched=launched, eos_exit=self.eos_exit)
