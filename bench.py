@@ -417,6 +417,78 @@ def time_lmhead(cfg, device, reps=10):
     return out, flops, hid, V * hid * 2 + rows * hid * 2
 
 
+def time_decode_loop(device, n_blocks=8, lookaheads=(0, 2)):
+    """The whole block-wise procedure on the LLaDA-shaped configuration (8 sequences, 32 layers, prompt 1024,
+    n_blocks blocks of 32): per block one refresh iteration (dense attention over prefix + retained rows, every
+    layer) and pruned iterations until the block has no mask left, driven by decode.BlockDecoder.  The model's
+    other layers are absent: the logits of an iteration come from a small pool of seeded buffers.  Compares the
+    synchronous loop (lookahead 0) with the host running ahead of the device."""
+    import torch
+    import paper_2601_17917_b200 as ds
+    from paper_2601_17917_b200 import workloads as wl
+    from paper_2601_17917_b200.decode import BlockDecoder
+    base = wl.CONFIGS["llada8x32"]
+    cfg = wl.shrink(base, gen=n_blocks * base.K, name="llada8x32-decode")
+    B, K, L, P, D = cfg.B, cfg.K, cfg.gen, cfg.P, cfg.D
+    layers = [wl.attention_inputs(cfg, device=device, layer=l) for l in range(cfg.n_layers)]
+    pool = [wl.logits(cfg, device=device, step=s, spike_range=(14.0, 26.0)) for s in range(4)]
+    scale = 1.0 / math.sqrt(D)
+    Lq_max = len(ds.retained_indices(L, K, 0, cfg.w, cfg.keep_last))
+    dt = cfg.torch_dtype()
+    # refresh iteration: queries and keys are all of prefix + retained rows (one seeded set shared by the layers)
+    ref_cfg = wl.shrink(cfg, P=0, gen=P + Lq_max, name="refresh")
+    dense = wl.attention_inputs(ref_cfg, device=device, layer=99)
+    out = torch.empty((B, cfg.Hq, P + Lq_max, D), dtype=dt, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    ar = torch.arange(P + Lq_max, dtype=torch.int32, device=device)
+
+    def forward_for(dec):
+        # the calls of a block repeat with the same pointers: plan them once per block
+        plans = {}
+
+        def forward(st):
+            key = (st.n, st.refresh)
+            if key not in plans:
+                if st.refresh:
+                    n_rows = P + len(ds.retained_indices(L, K, st.n, cfg.w, cfg.keep_last))
+                    one = ds.AttnPlan(dense["q_tail"], dense["k_tail"], dense["v_tail"], None, None, ar[:n_rows], scale,
+                                      out=out[:, :, :n_rows], status=status, seq_list=st.active_seq, n_seq=B,
+                                      n_seq_dev=st.active_cnt)
+                    plans[key] = [one] * cfg.n_layers
+                else:
+                    r0 = st.n * K
+                    plans[key] = [ds.AttnPlan(x["q_tail"][:, :, r0:], x["k_tail"][:, :, r0:], x["v_tail"][:, :, r0:],
+                                              x["k_pre"], x["v_pre"], st.idx, scale, out=out[:, :, :st.idx.numel()],
+                                              status=status, seq_list=st.active_seq, n_seq=B, n_seq_dev=st.active_cnt)
+                                  for x in layers]
+            for pl in plans[key]:
+                pl.launch()
+            return pool[(st.n + st.t) % len(pool)]
+        return forward
+
+    res = {"what": "whole block-wise decode (refresh + pruned iterations per block, early exit off); not part of `value`",
+           "workload": cfg.name, "blocks": n_blocks, "B": B, "K": K, "n_layers": cfg.n_layers, "runs": {}}
+    for la in lookaheads:
+        dec = BlockDecoder(B, L, K, cfg.V, tau0=cfg.tau0, alpha=cfg.alpha, mask_id=cfg.V - 1, w_tokens=cfg.w,
+                           keep_last=cfg.keep_last, device=device, lookahead=la)
+        forward = forward_for(dec)
+        dec.decode(forward)                       # warm-up (and the plans)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = ds.ds_launch_count()
+        a.record()
+        got = dec.decode(forward)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b)
+        res["runs"][f"lookahead{la}"] = {"ms": ms, "iterations": int(sum(got["steps"])),
+                                         "iterations_enqueued": int(sum(got["launched"])),
+                                         "ms_per_iteration": ms / max(1, sum(got["steps"])),
+                                         "launches": int(ds.ds_launch_count() - n0)}
+    res["device_status"] = int(ds.ds_read_status(status))
+    return res
+
+
 def time_rope(cfg, device, reps=20):
     """The widened path: rotary encoding + gather of the retained rows (ds_rope_gather), timed alone."""
     import torch
@@ -484,6 +556,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the extra timing of ds_lmhead_confidence")
+    ap.add_argument("--no-decode-loop", action="store_true", help="skip the extra timing of the block-wise decode loop")
     ap.add_argument("--stages", default="attn,confidence,select",
                     help="comma list of the stages a step runs (profiling a single kernel)")
     ap.add_argument("--vocab", type=int, default=0, help="override the vocabulary size (small profiler cases)")
@@ -632,6 +705,11 @@ def main():
                          "traffic": None},
             "weight_stream_gbs": in_bytes / (t["fused"] * 1e-3) / 1e9,
             "unfused_ms": t["unfused"], "unfused": "torch.matmul (library GEMM) to bf16 logits + ds_confidence"}
+    if not args.no_decode_loop and world == 1 and args.stages == "attn,confidence,select":
+        step = None
+        torch.cuda.empty_cache()
+        line["decode_loop"] = time_decode_loop(device)
+        torch.cuda.empty_cache()
     if not args.no_cpu_baseline and world == 1:
         smp = OracleSample(cfg, 32, 128)
         full_s, spent = smp.time()

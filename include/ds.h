@@ -131,6 +131,21 @@ DS_API size_t ds_attn_pruned_workspace(const ds_attn_params *p);
 /* `p` is a HOST pointer; the pointers inside it are device pointers. */
 DS_API int ds_attn_pruned(const ds_attn_params *p, void *stream);
 
+/* The same call split in two for loops that repeat it: within a block every iteration runs the attention of
+ * a layer on the same buffers, with the same retained rows (Eq. 7 depends on the block, not on the
+ * iteration), and only the device-resident sequence list changes.  ds_attn_plan_create validates *p, chooses
+ * the kernel and works out its parameters (tensor-map encodings included) once; ds_attn_plan_launch enqueues
+ * that kernel on `stream` and does nothing else, so its host cost is that of one kernel launch.  The plan
+ * (HOST memory, owned by the caller until ds_attn_plan_destroy) keeps the pointers of *p, not the memory
+ * behind them: every buffer must stay valid and in place while the plan is used; what the buffers, the
+ * index list, the sequence list and *n_seq_dev contain is read at each launch.  Launches of one plan may be
+ * captured into a CUDA graph.  A plan belongs to the device that was current when it was created.
+ * Errors of create: those of ds_attn_pruned; *plan is NULL on failure.  Destroying NULL is allowed. */
+typedef struct ds_attn_plan ds_attn_plan;
+DS_API int ds_attn_plan_create(const ds_attn_params *p, ds_attn_plan **plan);
+DS_API int ds_attn_plan_launch(const ds_attn_plan *plan, void *stream);
+DS_API void ds_attn_plan_destroy(ds_attn_plan *plan);
+
 /* ------------------------------------------------------------------------
  * ds_confidence  (Eq. 4)
  *
@@ -294,7 +309,9 @@ DS_API int ds_confidence_static(const void *logits, int32_t dtype, int64_t rows,
  * active_seq) restricts processing; NULL = all B.  With seq_list, n_seq may be
  * given as a device scalar instead (n_seq_dev != NULL overrides n_seq as the
  * count, n_seq then being only the upper bound used to size the launch).
- * Unprocessed sequences' outputs are left untouched.
+ * Unprocessed sequences' outputs are left untouched.  active_seq may be the same array as seq_list and
+ * active_cnt the same word as n_seq_dev (the list is then updated in place, which keeps the pointers of a
+ * loop's calls fixed); no other two arguments may overlap.
  * ------------------------------------------------------------------------ */
 typedef struct {
   int32_t B, K;                 /* 1 <= K <= 4096 */

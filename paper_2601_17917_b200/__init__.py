@@ -20,7 +20,8 @@ __all__ = [
     "lib", "retained_indices", "ds_attn_pruned", "ds_attn_pruned_workspace", "ds_confidence",
     "ds_confidence_workspace", "ds_confidence_static", "ds_lmhead_confidence", "ds_lmhead_confidence_workspace",
     "ds_rope_gather", "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
-    "ds_launch_count", "ds_block_begin", "ds_confidence_listed", "DsError", "DS_F32", "DS_BF16", "DS_DEV_INDEX", "DS_DEV_TIMEOUT",
+    "ds_launch_count", "ds_block_begin", "ds_confidence_listed", "AttnPlan",
+    "DsError", "DS_F32", "DS_BF16", "DS_DEV_INDEX", "DS_DEV_TIMEOUT",
 ]
 
 DS_F32, DS_BF16 = 0, 1
@@ -101,6 +102,12 @@ def lib() -> ctypes.CDLL:
         L.ds_attn_pruned_workspace.argtypes = [ctypes.POINTER(_AttnParams)]
         L.ds_attn_pruned.restype = ctypes.c_int
         L.ds_attn_pruned.argtypes = [ctypes.POINTER(_AttnParams), ctypes.c_void_p]
+        L.ds_attn_plan_create.restype = ctypes.c_int
+        L.ds_attn_plan_create.argtypes = [ctypes.POINTER(_AttnParams), ctypes.POINTER(ctypes.c_void_p)]
+        L.ds_attn_plan_launch.restype = ctypes.c_int
+        L.ds_attn_plan_launch.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+        L.ds_attn_plan_destroy.restype = None
+        L.ds_attn_plan_destroy.argtypes = [ctypes.c_void_p]
         L.ds_confidence_workspace.restype = ctypes.c_size_t
         L.ds_confidence_workspace.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int32]
         L.ds_confidence.restype = ctypes.c_int
@@ -260,6 +267,45 @@ def ds_attn_pruned(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out=N
     if rc != DS_OK:
         raise DsError(rc, "ds_attn_pruned")
     return out
+
+
+class AttnPlan:
+    """ds_attn_plan: the arguments of ds_attn_pruned validated and turned into kernel parameters once;
+    ``launch`` then only enqueues the kernel.  The plan keeps references to the tensors it was made from
+    (their contents are read at every launch).  ``out`` is allocated when not given."""
+
+    def __init__(self, q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out=None, lse=None, workspace=None,
+                 status=None, seq_list=None, n_seq=None, n_seq_dev=None):
+        _check_dev(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, out, lse, workspace, status, seq_list, n_seq_dev)
+        B, Hq, T, D = q_tail.shape
+        if out is None:
+            out = torch.empty((B, Hq, idx.shape[-1], D), dtype=q_tail.dtype, device=q_tail.device)
+        p = _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status,
+                         seq_list, n_seq, n_seq_dev)
+        if workspace is None:
+            need = int(lib().ds_attn_pruned_workspace(ctypes.byref(p)))
+            if need:
+                workspace = torch.empty(need, dtype=torch.uint8, device=q_tail.device)
+                p.workspace, p.workspace_bytes = workspace.data_ptr(), need
+        self.out = out
+        self._keep = (q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, out, lse, workspace, status, seq_list, n_seq_dev)
+        self._h = ctypes.c_void_p()
+        self._destroy = lib().ds_attn_plan_destroy
+        self._launch = lib().ds_attn_plan_launch
+        rc = lib().ds_attn_plan_create(ctypes.byref(p), ctypes.byref(self._h))
+        if rc != DS_OK:
+            raise DsError(rc, "ds_attn_plan_create")
+
+    def launch(self, stream=None):
+        rc = self._launch(self._h, _stream(stream))
+        if rc != DS_OK:
+            raise DsError(rc, "ds_attn_plan_launch")
+        return self.out
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            self._destroy(h)
 
 
 def ds_confidence_workspace(rows: int, V: int, dtype) -> int:

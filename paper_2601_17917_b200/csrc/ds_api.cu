@@ -3,6 +3,7 @@
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
+#include <new>
 
 #include "ds_common.cuh"
 
@@ -82,27 +83,74 @@ size_t ds_attn_pruned_workspace(const ds_attn_params *p) {
   return 0;
 }
 
-int ds_attn_pruned(const ds_attn_params *p, void *stream) {
-  const int rc = ds::validate_attn(p);
+namespace ds {
+namespace {
+// Validation, choice of the kernel and its parameters for one set of arguments.
+int resolve_attn(const ds_attn_params *p, AttnPrepared &a) {
+  const int rc = validate_attn(p);
   if (rc != DS_OK) return rc;
+  a.p = *p;
+  a.grid = 0;
+  a.path = kAttnPathSimt;
   if (p->B == 0) return DS_OK;
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  const ds::AttnPath path = ds::forced_path();
-  const bool tc_ok = ds::attn_tc_supported(*p);
-  if ((path == ds::AttnPath::kTc || path == ds::AttnPath::kTc2) && !tc_ok) return DS_ERR_UNSUPPORTED;
-  if (tc_ok && path == ds::AttnPath::kTc2) return ds::launch_attn_tc2(*p, st);
-  if (tc_ok && path != ds::AttnPath::kSimt) {
-    const size_t need = ds::attn_tc_workspace_bytes(*p);
-    if (need > 0 && (!p->workspace || !ds::aligned(p->workspace, 256) || p->workspace_bytes < need))
-      return DS_ERR_WORKSPACE;
-    // Many M-tiles per KV head (the unpruned reference, a cache-refresh step): the two-tile kernel shares every
-    // KV tile between two M-tiles; measured faster from about 8 tile pairs on, slower below.
-    const long long stacked_rows = (long long)(p->Hq / p->Hkv) * p->Lq;
-    if (path == ds::AttnPath::kAuto && stacked_rows >= 2048) return ds::launch_attn_tc2(*p, st);
-    return ds::launch_attn_tc(*p, st);
+  const AttnPath path = forced_path();
+  const bool tc_ok = attn_tc_supported(*p);
+  if ((path == AttnPath::kTc || path == AttnPath::kTc2) && !tc_ok) return DS_ERR_UNSUPPORTED;
+  if (tc_ok && path == AttnPath::kTc2) return prepare_attn_tc2(*p, a);
+  if (tc_ok && path != AttnPath::kSimt) {
+    const size_t need = attn_tc_workspace_bytes(*p);
+    if (need > 0 && (!p->workspace || !aligned(p->workspace, 256) || p->workspace_bytes < need)) return DS_ERR_WORKSPACE;
+    // The two-tile kernel (one KV tile shared by two M-tiles) stays selectable through DS_ATTN_PATH=tc2 but is
+    // not dispatched: once consecutive retained rows are fetched as whole-tile boxes the one-tile kernel is
+    // the faster one on every measured shape, pruned or dense.
+    return prepare_attn_tc(*p, a);
   }
-  return ds::launch_attn_simt(*p, st);
+  a.grid = 1;  // the SIMT launcher sizes its own grid from a.p
+  return DS_OK;
 }
+
+int launch_resolved(const AttnPrepared &a, cudaStream_t st) {
+  if (a.p.B == 0) return DS_OK;
+  switch (a.path) {
+    case kAttnPathTc: return launch_prepared_tc(a, st);
+    case kAttnPathTc2: return launch_prepared_tc2(a, st);
+    default: return launch_attn_simt(a.p, st);
+  }
+}
+}  // namespace
+}  // namespace ds
+
+struct ds_attn_plan {
+  ds::AttnPrepared a;
+};
+
+int ds_attn_pruned(const ds_attn_params *p, void *stream) {
+  ds::AttnPrepared a;
+  const int rc = ds::resolve_attn(p, a);
+  if (rc != DS_OK) return rc;
+  return ds::launch_resolved(a, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int ds_attn_plan_create(const ds_attn_params *p, ds_attn_plan **plan) {
+  if (!plan) return DS_ERR_INVALID_ARG;
+  *plan = nullptr;
+  ds_attn_plan *pl = new (std::nothrow) ds_attn_plan;
+  if (!pl) return DS_ERR_CUDA;
+  const int rc = ds::resolve_attn(p, pl->a);
+  if (rc != DS_OK) {
+    delete pl;
+    return rc;
+  }
+  *plan = pl;
+  return DS_OK;
+}
+
+int ds_attn_plan_launch(const ds_attn_plan *plan, void *stream) {
+  if (!plan) return DS_ERR_INVALID_ARG;
+  return ds::launch_resolved(plan->a, reinterpret_cast<cudaStream_t>(stream));
+}
+
+void ds_attn_plan_destroy(ds_attn_plan *plan) { delete plan; }
 
 size_t ds_confidence_workspace(int64_t rows, int64_t V, int32_t dtype) {
   if (dtype != DS_F32 && dtype != DS_BF16) return 0;

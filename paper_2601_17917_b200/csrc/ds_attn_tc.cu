@@ -52,6 +52,7 @@
 #include <cstring>
 #include <mutex>
 
+
 #include "ds_attn_tiles.cuh"
 #include "ds_common.cuh"
 #include "ds_sm100.cuh"
@@ -225,6 +226,9 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       prefetch_map(&prm.v1);
       prefetch_map(&prm.q32);
       prefetch_map(&prm.q1);
+      prefetch_map(&prm.k128);
+      prefetch_map(&prm.v128);
+      prefetch_map(&prm.q128);
     }
     // one index list for all batches: keep (the head of) it in shared memory, validated once
     const int32_t *idx_cache = nullptr;
@@ -247,14 +251,14 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     // item's last Q K^T has completed.
     auto issue_q = [&](int kq) {
       const Item it = decode_item(prm, blockIdx.x + kq * gridDim.x);
-      uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
+      uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
                                       it.mt * kBlockM, it.m_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
       if (it.x_rows > 0) {
         // rows of the small query tile that are not loaded must be finite: clear the tile first
         for (int q = lane; q < (2 * kXChunkBytes) / 16; q += 32)
           *reinterpret_cast<uint4 *>(smem + G_::kOffQx + q * 16) = make_uint4(0, 0, 0, 0);
         fence_proxy_async();
-        bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, sbase + G_::kOffQx, kXChunkBytes, bar_q_full,
+        bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQx, kXChunkBytes, bar_q_full,
                                 (it.mt + 1) * kBlockM, it.x_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
       }
       if (lane == 0) mbar_arrive_expect_tx(bar_q_full, bytes);
@@ -322,7 +326,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
               fence_proxy_async();
             }
             // the V fill of a tile directly follows its K fill: the staged row list is still valid
-            const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, dst, kChunkBytes,
+            const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, kv ? &prm.v128 : &prm.k128, dst, kChunkBytes,
                                                   full, t0, n, it.hk, it.b, idx_s, idx_cache, bad_index, kv == 1);
             if (lane == 0) mbar_arrive_expect_tx(full, bytes);
           }
@@ -808,11 +812,13 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
 // Host side
 // ------------------------------------------------------------------------------------------------
 template <int D>
-int launch_d(const ds_attn_params &p, cudaStream_t stream) {
-  // the attribute is per device: set it at every launch (cheap)
-  DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes));
-  TcParams prm;
+int prepare_d(const ds_attn_params &p, AttnPrepared &out) {
+  static_assert(sizeof(TcParams) <= sizeof(out.kernel_params), "parameter struct does not fit the plan");
+  TcParams &prm = *reinterpret_cast<TcParams *>(out.kernel_params);  // plain data, zeroed below
   memset(&prm, 0, sizeof(prm));
+  out.path = kAttnPathTc;
+  out.p = p;
+  out.grid = 0;
   if (!fill_common(prm, p)) return DS_ERR_CUDA;
   // stacked query rows of one KV head: full 128-row tiles, and a remainder that either rides along
   // with the last full tile (1..kXMax rows, D = 128) or gets a tile of its own
@@ -828,9 +834,16 @@ int launch_d(const ds_attn_params &p, cudaStream_t stream) {
   const long long n_items = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv * prm.n_mtiles;  // upper bound with a device count
   if (n_items > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   prm.n_items = (int)n_items;
-  if (n_items == 0) return DS_OK;
-  const int grid = (int)(n_items < sm_count() ? n_items : sm_count());
-  attn_tc_kernel<D><<<grid, kNumThreads, Geo<D>::kSmemBytes, stream>>>(prm);
+  out.grid = (int)(n_items < sm_count() ? n_items : sm_count());
+  return DS_OK;
+}
+
+template <int D>
+int launch_prepared_d(const AttnPrepared &a, cudaStream_t stream) {
+  if (a.grid == 0) return DS_OK;
+  // the attribute is per device: set it at every launch (cheap)
+  DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes));
+  attn_tc_kernel<D><<<a.grid, kNumThreads, Geo<D>::kSmemBytes, stream>>>(*reinterpret_cast<const TcParams *>(a.kernel_params));
   DS_CUDA_OK(cudaGetLastError());
   note_launch(1);
   return DS_OK;
@@ -870,6 +883,9 @@ bool fill_common(AttnCommon &c, const ds_attn_params &p) {
   ok = ok && make_map(&c.v1, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 1);
   ok = ok && make_map(&c.q32, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 32);
   ok = ok && make_map(&c.q1, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 1);
+  ok = ok && make_map(&c.k128, p.k_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 128);
+  ok = ok && make_map(&c.v128, p.v_tail, D, p.T, p.Hkv, p.B, p.kv_tail_stride, 128);
+  ok = ok && make_map(&c.q128, p.q_tail, D, p.T, p.Hq, p.B, p.q_stride, 128);
   if (!ok) return false;
   c.idx = p.idx;
   c.idx_bstride = p.idx_batch_stride;
@@ -919,8 +935,16 @@ bool attn_tc_supported(const ds_attn_params &p) {
 
 size_t attn_tc_workspace_bytes(const ds_attn_params &) { return 0; }
 
+int prepare_attn_tc(const ds_attn_params &p, AttnPrepared &out) {
+  return p.D == 128 ? prepare_d<128>(p, out) : prepare_d<64>(p, out);
+}
+int launch_prepared_tc(const AttnPrepared &a, cudaStream_t stream) {
+  return a.p.D == 128 ? launch_prepared_d<128>(a, stream) : launch_prepared_d<64>(a, stream);
+}
 int launch_attn_tc(const ds_attn_params &p, cudaStream_t stream) {
-  return p.D == 128 ? launch_d<128>(p, stream) : launch_d<64>(p, stream);
+  AttnPrepared a;
+  const int rc = prepare_attn_tc(p, a);
+  return rc != DS_OK ? rc : launch_prepared_tc(a, stream);
 }
 
 }  // namespace ds

@@ -24,6 +24,7 @@
 
 #include <cstring>
 
+
 #include "ds_attn_tiles.cuh"
 #include "ds_common.cuh"
 #include "ds_sm100.cuh"
@@ -147,6 +148,9 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
       prefetch_map(&prm.v1);
       prefetch_map(&prm.q32);
       prefetch_map(&prm.q1);
+      prefetch_map(&prm.k128);
+      prefetch_map(&prm.v128);
+      prefetch_map(&prm.q128);
     }
     const int32_t *idx_cache = nullptr;
     if (prm.idx_bstride == 0) {
@@ -166,10 +170,10 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
     int q_next = 0;
     auto issue_q = [&](int kq) {
       const Item2 it = decode_item2(prm, blockIdx.x + kq * gridDim.x);
-      uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
+      uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
                                       it.pr * 2 * kBlockM, it.rows_a, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
       if (it.rows_b > 0)
-        bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, sbase + G_::kOffQ + G_::kTileBytes, kChunkBytes, bar_q_full,
+        bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ + G_::kTileBytes, kChunkBytes, bar_q_full,
                                 (it.pr * 2 + 1) * kBlockM, it.rows_b, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
       if (lane == 0) mbar_arrive_expect_tx(bar_q_full, bytes);
     };
@@ -229,7 +233,7 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
               }
               fence_proxy_async();
             }
-            const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, dst, kChunkBytes,
+            const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, kv ? &prm.v128 : &prm.k128, dst, kChunkBytes,
                                                   full, t0, n, it.hk, it.b, idx_s, idx_cache, bad_index, kv == 1);
             if (lane == 0) mbar_arrive_expect_tx(full, bytes);
           }
@@ -478,19 +482,28 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
 }
 
 template <int D>
-int launch2_d(const ds_attn_params &p, cudaStream_t stream) {
-  DS_CUDA_OK(cudaFuncSetAttribute(attn_tc2_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo2<D>::kSmemBytes));
-  Tc2Params prm;
+int prepare2_d(const ds_attn_params &p, AttnPrepared &out) {
+  static_assert(sizeof(Tc2Params) <= sizeof(out.kernel_params), "parameter struct does not fit the plan");
+  Tc2Params &prm = *reinterpret_cast<Tc2Params *>(out.kernel_params);  // plain data, zeroed below
   memset(&prm, 0, sizeof(prm));
+  out.path = kAttnPathTc2;
+  out.p = p;
+  out.grid = 0;
   if (!fill_common(prm, p)) return DS_ERR_CUDA;
   const long long rows_total = (long long)prm.G * p.Lq;
   prm.n_pairs = (int)((rows_total + 2 * kBlockM - 1) / (2 * kBlockM));
   const long long n_items = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv * prm.n_pairs;  // upper bound with a device count
   if (n_items > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   prm.n_items = (int)n_items;
-  if (n_items == 0) return DS_OK;
-  const int grid = (int)(n_items < sm_count() ? n_items : sm_count());
-  attn_tc2_kernel<D><<<grid, kThreads2, Geo2<D>::kSmemBytes, stream>>>(prm);
+  out.grid = (int)(n_items < sm_count() ? n_items : sm_count());
+  return DS_OK;
+}
+
+template <int D>
+int launch_prepared2_d(const AttnPrepared &a, cudaStream_t stream) {
+  if (a.grid == 0) return DS_OK;
+  DS_CUDA_OK(cudaFuncSetAttribute(attn_tc2_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo2<D>::kSmemBytes));
+  attn_tc2_kernel<D><<<a.grid, kThreads2, Geo2<D>::kSmemBytes, stream>>>(*reinterpret_cast<const Tc2Params *>(a.kernel_params));
   DS_CUDA_OK(cudaGetLastError());
   note_launch(1);
   return DS_OK;
@@ -498,8 +511,16 @@ int launch2_d(const ds_attn_params &p, cudaStream_t stream) {
 
 }  // namespace
 
+int prepare_attn_tc2(const ds_attn_params &p, AttnPrepared &out) {
+  return p.D == 128 ? prepare2_d<128>(p, out) : prepare2_d<64>(p, out);
+}
+int launch_prepared_tc2(const AttnPrepared &a, cudaStream_t stream) {
+  return a.p.D == 128 ? launch_prepared2_d<128>(a, stream) : launch_prepared2_d<64>(a, stream);
+}
 int launch_attn_tc2(const ds_attn_params &p, cudaStream_t stream) {
-  return p.D == 128 ? launch2_d<128>(p, stream) : launch2_d<64>(p, stream);
+  AttnPrepared a;
+  const int rc = prepare_attn_tc2(p, a);
+  return rc != DS_OK ? rc : launch_prepared_tc2(a, stream);
 }
 
 }  // namespace ds

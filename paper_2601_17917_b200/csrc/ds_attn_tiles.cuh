@@ -16,6 +16,7 @@ constexpr int kIdxCap = 2048;           // entries of a shared index list kept i
 
 struct AttnCommon {
   CUtensorMap kpre, vpre, k32, k1, v32, v1, q32, q1;
+  CUtensorMap k128, v128, q128;  // boxes of a whole 128-row tile, for runs of consecutive rows
   const int32_t *idx;
   long long idx_bstride;
   void *out;
@@ -59,7 +60,7 @@ __device__ __forceinline__ bool bad_sequence_numbers(const AttnCommon &c, int n_
 // ------------------------------------------------------------------------------------------------
 template <int D>
 __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUtensorMap *map32, const CUtensorMap *map1,
-                                                uint32_t dst, uint32_t chunk_stride, uint32_t bar, int R0, int n,
+                                                const CUtensorMap *map128, uint32_t dst, uint32_t chunk_stride, uint32_t bar, int R0, int n,
                                                 int head0, int b, int32_t *idx_s, const int32_t *idx_cache,
                                                 bool &bad_index, bool staged = false) {
   const int lane = threadIdx.x & 31;
@@ -92,6 +93,14 @@ __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUt
   }
   uint32_t bytes = 0;
   if (lane == 0) {
+    // a full tile of consecutive rows inside one head (the current block and its window, every tile of a
+    // cache-refresh step): one box per 64-column chunk.  The list is strictly ascending, so first and last
+    // entry decide.
+    if (n == 128 && pos0 + 128 <= Lq && idx_s[127] - idx_s[0] == 127) {
+#pragma unroll
+      for (int c = 0; c < (D / 64); ++c) tma_load_4d(dst + c * chunk_stride, map128, bar, c * 64, idx_s[0], head, b);
+      return 128u * 128u * (D / 64);
+    }
     int r = 0, pos = pos0;
     while (r < n) {
       const int row = idx_s[r];

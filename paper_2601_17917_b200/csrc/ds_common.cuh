@@ -55,6 +55,20 @@ int launch_rope_gather(const ds_rope_params &p, cudaStream_t stream);
 int launch_attn_simt(const ds_attn_params &p, cudaStream_t stream);
 int launch_attn_tc(const ds_attn_params &p, cudaStream_t stream);
 int launch_attn_tc2(const ds_attn_params &p, cudaStream_t stream);
+
+// An attention call whose kernel parameters (tensor maps included) have been worked out once: what a
+// ds_attn_plan holds and what the one-shot launchers build on the stack.
+enum : int { kAttnPathSimt = 0, kAttnPathTc = 1, kAttnPathTc2 = 2 };
+struct AttnPrepared {
+  int path;
+  int grid;          // CTAs to launch; 0 = nothing to do
+  ds_attn_params p;  // validated copy of the caller's arguments (the SIMT kernel takes it as it is)
+  alignas(64) unsigned char kernel_params[2048];  // the tensor-core kernels' parameter struct
+};
+int prepare_attn_tc(const ds_attn_params &p, AttnPrepared &out);
+int prepare_attn_tc2(const ds_attn_params &p, AttnPrepared &out);
+int launch_prepared_tc(const AttnPrepared &a, cudaStream_t stream);
+int launch_prepared_tc2(const AttnPrepared &a, cudaStream_t stream);
 bool attn_tc_supported(const ds_attn_params &p);
 size_t attn_tc_workspace_bytes(const ds_attn_params &p);
 

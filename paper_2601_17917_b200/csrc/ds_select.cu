@@ -108,7 +108,9 @@ __device__ __forceinline__ int listed_count(const ds_select_params &p) {
 }
 
 // Ordered compaction of the processed sequences whose block is not finished.
-// Runs in one CTA of kSelThreads threads.
+// Runs in one CTA of kSelThreads threads.  active_seq may be the array seq_list points to and active_cnt the
+// word n_seq_dev points to: every thread has read its entry of a round (and the count) before the barrier
+// that precedes the round's writes, and a round only writes positions at or below the ones it read.
 __device__ void compact_active(const ds_select_params &p, int n) {
   __shared__ int warp_cnt[kSelWarps];
   __shared__ int running;
@@ -121,7 +123,7 @@ __device__ void compact_active(const ds_select_params &p, int n) {
     bool act = false;
     if (s < n) {
       b = p.seq_list ? p.seq_list[s] : s;
-      act = p.block_done[b] == 0;
+      act = (b >= 0 && b < p.B) && p.block_done[b] == 0;
     }
     const unsigned bal = __ballot_sync(0xffffffffu, act);
     if (lane == 0) warp_cnt[wid] = __popc(bal);
@@ -196,8 +198,9 @@ __global__ void __launch_bounds__(kSelThreads) select_fused_kernel(const ds_sele
     if (b >= 0 && b < p.B) select_sequence(p, b, lane);
   }
   __syncthreads();  // block_done and the mask flags of every sequence written by this CTA are visible below
-  compact_active(p, n);
+  // the row list first: it walks seq_list, which compact_active may overwrite (active_seq may be the same array)
   if (p.masked_rows != nullptr) compact_masked_rows(p, n);
+  compact_active(p, n);
 }
 
 __global__ void __launch_bounds__(256) select_grid_kernel(const ds_select_params p) {
@@ -211,8 +214,8 @@ __global__ void __launch_bounds__(256) select_grid_kernel(const ds_select_params
 
 __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const ds_select_params p) {
   const int n = listed_count(p);
-  compact_active(p, n);
   if (p.masked_rows != nullptr) compact_masked_rows(p, n);
+  compact_active(p, n);
 }
 
 // Start of a block: mask flags, block tokens and the lists of the sequences that have not exited.

@@ -12,7 +12,8 @@ iterations per block are enqueued, and they find empty lists and do nothing.
 
 The model itself (Eq. 3) is the caller's: ``forward(step)`` must leave the logits of the current block's
 positions in ``step.logits`` using ``step.idx`` (retained rows, Eq. 7), ``step.refresh`` (first iteration of
-a block: every position is a query and the prefix cache is rebuilt) and the device lists.
+a block: every position is a query and the prefix cache is rebuilt) and the device lists; it may instead
+return a tensor of the same shape and type that already holds them.
 """
 from __future__ import annotations
 
@@ -57,17 +58,16 @@ class BlockDecoder:
         self.tok = torch.zeros(B * K, **i32)
         self.logits = torch.zeros((B * K, V), dtype=logits_dtype, device=dev)
         self.eos_exit = torch.zeros(B, dtype=torch.uint8, device=dev)
-        # the active list is read and rewritten by the same selection kernel: two copies, used alternately
-        self.active = [torch.zeros(max(B, 1), **i32) for _ in range(2)]
-        self.active_cnt = [torch.zeros(1, **i32) for _ in range(2)]
-        self.sel = [dict(sel_idx=torch.empty((B, K), **i32), sel_cnt=torch.zeros(B, **i32),
-                         block_done=torch.zeros(B, dtype=torch.uint8, device=dev), eos_exit=self.eos_exit,
-                         active_seq=self.active[k], active_cnt=self.active_cnt[k],
-                         masked_rows=None, masked_cnt=None) for k in range(2)]
+        # the selection updates the active list in place: every call of the loop sees the same pointers, so
+        # attention plans (and CUDA graphs of an iteration) made once stay valid for the whole block
+        self.active = torch.zeros(max(B, 1), **i32)
+        self.active_cnt = torch.zeros(1, **i32)
         self.masked_rows = torch.zeros(max(B * K, 1), **i32)
         self.masked_cnt = torch.zeros(1, **i32)
-        for s in self.sel:
-            s["masked_rows"], s["masked_cnt"] = self.masked_rows, self.masked_cnt
+        self.sel = dict(sel_idx=torch.empty((B, K), **i32), sel_cnt=torch.zeros(B, **i32),
+                        block_done=torch.zeros(B, dtype=torch.uint8, device=dev), eos_exit=self.eos_exit,
+                        active_seq=self.active, active_cnt=self.active_cnt,
+                        masked_rows=self.masked_rows, masked_cnt=self.masked_cnt)
         self.workspace = torch.empty(max(ds_confidence_workspace(B * K, V, logits_dtype), 1), dtype=torch.uint8,
                                      device=dev)
         # Eq. 7 per block: the retained rows of the pruned iterations and all rows for the refresh iteration
@@ -93,28 +93,30 @@ class BlockDecoder:
         self.eos_exit.zero_()
         steps, launched = [], []
         for n in range(N):
-            ds_block_begin(self.eos_exit, self.masked, self.x_block, self.mask_id, self.eos_id, self.active[0],
-                           self.active_cnt[0], self.masked_rows, self.masked_cnt)
-            self._publish(0, self.active_cnt[0])
-            cur, t = 0, 0
+            ds_block_begin(self.eos_exit, self.masked, self.x_block, self.mask_id, self.eos_id, self.active,
+                           self.active_cnt, self.masked_rows, self.masked_cnt)
+            self._publish(0, self.active_cnt)
+            t = 0
             while t < K:
                 seen = t - self.lookahead            # the newest slot the host insists on having seen
                 if seen >= 0:
                     self.events[seen].synchronize()
                     if int(self.cnt_host[seen]) == 0:
                         break
-                forward(Step(n=n, t=t, refresh=(t == 0), idx=self.idx_all[n] if t == 0 else self.idx[n],
-                             active_seq=self.active[cur], active_cnt=self.active_cnt[cur], x_block=self.x_block,
-                             logits=self.logits))
-                ds_confidence_listed(self.logits, self.masked_rows, self.masked_cnt, self.conf, self.tok,
+                z = forward(Step(n=n, t=t, refresh=(t == 0), idx=self.idx_all[n] if t == 0 else self.idx[n],
+                                 active_seq=self.active, active_cnt=self.active_cnt, x_block=self.x_block,
+                                 logits=self.logits))
+                if z is None:
+                    z = self.logits
+                elif z.shape != self.logits.shape or z.dtype != self.logits.dtype or z.device != self.logits.device:
+                    raise ValueError("forward returned logits of the wrong shape, type or device")
+                ds_confidence_listed(z, self.masked_rows, self.masked_cnt, self.conf, self.tok,
                                      n_listed_max=B * K, workspace=self.workspace)
                 ds_unmask_select(self.conf.view(B, K), self.tok.view(B, K), self.masked, self.x_block, self.tau0,
                                  self.alpha, ratio_extra=self.extra[n], eos_id=self.eos_id, eos_tau=self.eos_tau,
-                                 seq_list=self.active[cur], n_seq=B, n_seq_dev=self.active_cnt[cur],
-                                 out=self.sel[cur ^ 1])
-                cur ^= 1
+                                 seq_list=self.active, n_seq=B, n_seq_dev=self.active_cnt, out=self.sel)
                 t += 1
-                self._publish(t, self.active_cnt[cur])
+                self._publish(t, self.active_cnt)
             self.events[t].synchronize()             # everything enqueued for this block has run
             need = next(j for j in range(t + 1) if int(self.cnt_host[j]) == 0)
             steps.append(need)

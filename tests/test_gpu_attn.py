@@ -299,3 +299,37 @@ def test_listed_sequences_only(path, dtype, Lq, monkeypatch):
     ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, status=status, seq_list=bad)
     torch.cuda.synchronize()
     assert ds.ds_read_status(status) & ds.DS_DEV_INDEX
+
+
+@pytest.mark.parametrize("path,dtype", [("simt", torch.float32), ("tc", torch.bfloat16), ("tc2", torch.bfloat16)])
+def test_plan_launches_repeat_the_one_shot_call(path, dtype, monkeypatch):
+    monkeypatch.setenv("DS_ATTN_PATH", path)
+    B, Hq, Hkv, D, P, T, Lq = 3, 4, 2, 128, 150, 400, 261
+    g = torch.Generator().manual_seed(5)
+    mk = lambda *sh: torch.randn(*sh, generator=g).to(dtype).to(DEV)
+    q, kt, vt, kp, vp = mk(B, Hq, T, D), mk(B, Hkv, T, D), mk(B, Hkv, T, D), mk(B, Hkv, P, D), mk(B, Hkv, P, D)
+    idx = torch.arange(Lq, dtype=torch.int32, device=DEV)
+    scale = 1.0 / math.sqrt(D)
+    lst = torch.tensor([0, 2, 1], dtype=torch.int32, device=DEV)
+    cnt = torch.tensor([2], dtype=torch.int32, device=DEV)
+    plan = ds.AttnPlan(q, kt, vt, kp, vp, idx, scale, seq_list=lst, n_seq_dev=cnt)
+    n0 = ds.ds_launch_count()
+    plan.out.fill_(55.0)
+    plan.launch()
+    torch.cuda.synchronize()
+    assert ds.ds_launch_count() == n0 + 1
+    ref = oracle.attn(_np(q), _np(kt), _np(vt), _np(kp), _np(vp), idx.cpu().numpy(), scale)
+    _compare(plan.out[0], ref[0], dtype)
+    _compare(plan.out[2], ref[2], dtype)
+    assert (plan.out[1] == 55.0).all()
+    # what the buffers and the device-side list hold is read at every launch
+    cnt.fill_(3)
+    kt.copy_(mk(B, Hkv, T, D))
+    plan.launch()
+    torch.cuda.synchronize()
+    ref = oracle.attn(_np(q), _np(kt), _np(vt), _np(kp), _np(vp), idx.cpu().numpy(), scale)
+    for b in range(B):
+        _compare(plan.out[b], ref[b], dtype)
+    one_shot = ds.ds_attn_pruned(q, kt, vt, kp, vp, idx, scale)
+    assert torch.equal(one_shot, plan.out)
+    del plan

@@ -163,6 +163,38 @@ def test_seq_list_device_count_and_large_batch():
     assert g["active_seq"].tolist() == []
 
 
+@pytest.mark.parametrize("B", [40, 3000])
+def test_active_list_updated_in_place(B):
+    # active_seq aliases seq_list and active_cnt aliases n_seq_dev: the list shrinks in place over the steps
+    rng = np.random.default_rng(21)
+    K = 32
+    masked = np.ones((B, K), np.uint8)
+    x = np.full((B, K), -1, np.int32)
+    lst = torch.arange(B, dtype=torch.int32, device=DEV)
+    cnt = torch.tensor([B], dtype=torch.int32, device=DEV)
+    gm, gx = torch.tensor(masked, device=DEV), torch.tensor(x, device=DEV)
+    out = dict(sel_idx=torch.empty((B, K), dtype=torch.int32, device=DEV),
+               sel_cnt=torch.zeros(B, dtype=torch.int32, device=DEV),
+               block_done=torch.zeros(B, dtype=torch.uint8, device=DEV),
+               eos_exit=torch.zeros(B, dtype=torch.uint8, device=DEV), active_seq=lst, active_cnt=cnt,
+               masked_rows=torch.empty(B * K, dtype=torch.int32, device=DEV),
+               masked_cnt=torch.zeros(1, dtype=torch.int32, device=DEV))
+    active = list(range(B))
+    for step in range(6):
+        conf = rng.random((B, K)).astype(np.float32) ** 0.25
+        tok = rng.integers(0, 50, (B, K)).astype(np.int32)
+        o = oracle.select(conf, tok, masked, x, 0.9, 0.3, seq_list=active)
+        ds.ds_unmask_select(torch.tensor(conf, device=DEV), torch.tensor(tok, device=DEV), gm, gx, 0.9, 0.3,
+                            seq_list=lst, n_seq=B, n_seq_dev=cnt, out=out)
+        torch.cuda.synchronize()
+        masked, x, active = o["masked"], o["x_block"], o["active_seq"].tolist()
+        assert cnt.item() == len(active) and lst[:len(active)].cpu().tolist() == active
+        assert np.array_equal(gm.cpu().numpy(), masked) and np.array_equal(gx.cpu().numpy(), x)
+        want_rows = [b * K + i for b in range(B) for i in np.nonzero(masked[b])[0]]
+        assert out["masked_rows"][:out["masked_cnt"].item()].cpu().tolist() == want_rows
+    assert len(active) < B
+
+
 def _chain(cfg, steps, alpha, eos_id):
     """Config-4 style simulation: few masks per sequence, fresh logits each step."""
     x0, m0 = wl.block_state(cfg, "few")
