@@ -417,74 +417,80 @@ def time_lmhead(cfg, device, reps=10):
     return out, flops, hid, V * hid * 2 + rows * hid * 2
 
 
-def time_decode_loop(device, n_blocks=8, lookaheads=(0, 2)):
-    """The whole block-wise procedure on the LLaDA-shaped configuration (8 sequences, 32 layers, prompt 1024,
-    n_blocks blocks of 32): per block one refresh iteration (dense attention over prefix + retained rows, every
-    layer) and pruned iterations until the block has no mask left, driven by decode.BlockDecoder.  The model's
-    other layers are absent: the logits of an iteration come from a small pool of seeded buffers.  Compares the
-    synchronous loop (lookahead 0) with the host running ahead of the device."""
+def time_decode_loop(device, n_blocks=8, batches=(8, 1)):
+    """The whole block-wise procedure on the LLaDA-shaped configuration (32 layers, prompt 1024, n_blocks blocks
+    of 32; 8 sequences, and 1 as in the paper's per-sample latency figures): per block one refresh iteration
+    (dense attention over prefix + retained rows, every layer) and pruned iterations until the block has no mask
+    left, driven by decode.BlockDecoder.  The model's other layers are absent: the logits of an iteration are
+    staged from a small pool of seeded buffers.  Three ways to drive the same device work: the synchronous loop
+    (the host waits for every iteration), the host running two iterations ahead, and the latter with every
+    iteration replayed as one CUDA graph."""
     import torch
     import paper_2601_17917_b200 as ds
     from paper_2601_17917_b200 import workloads as wl
     from paper_2601_17917_b200.decode import BlockDecoder
     base = wl.CONFIGS["llada8x32"]
-    cfg = wl.shrink(base, gen=n_blocks * base.K, name="llada8x32-decode")
-    B, K, L, P, D = cfg.B, cfg.K, cfg.gen, cfg.P, cfg.D
-    layers = [wl.attention_inputs(cfg, device=device, layer=l) for l in range(cfg.n_layers)]
-    pool = [wl.logits(cfg, device=device, step=s, spike_range=(14.0, 26.0)) for s in range(4)]
-    scale = 1.0 / math.sqrt(D)
-    Lq_max = len(ds.retained_indices(L, K, 0, cfg.w, cfg.keep_last))
-    dt = cfg.torch_dtype()
-    # refresh iteration: queries and keys are all of prefix + retained rows (one seeded set shared by the layers)
-    ref_cfg = wl.shrink(cfg, P=0, gen=P + Lq_max, name="refresh")
-    dense = wl.attention_inputs(ref_cfg, device=device, layer=99)
-    out = torch.empty((B, cfg.Hq, P + Lq_max, D), dtype=dt, device=device)
-    status = torch.zeros(1, dtype=torch.int32, device=device)
-    ar = torch.arange(P + Lq_max, dtype=torch.int32, device=device)
-
-    def forward_for(dec):
-        # the calls of a block repeat with the same pointers: plan them once per block
-        plans = {}
-
-        def forward(st):
-            key = (st.n, st.refresh)
-            if key not in plans:
-                if st.refresh:
-                    n_rows = P + len(ds.retained_indices(L, K, st.n, cfg.w, cfg.keep_last))
-                    one = ds.AttnPlan(dense["q_tail"], dense["k_tail"], dense["v_tail"], None, None, ar[:n_rows], scale,
-                                      out=out[:, :, :n_rows], status=status, seq_list=st.active_seq, n_seq=B,
-                                      n_seq_dev=st.active_cnt)
-                    plans[key] = [one] * cfg.n_layers
-                else:
-                    r0 = st.n * K
-                    plans[key] = [ds.AttnPlan(x["q_tail"][:, :, r0:], x["k_tail"][:, :, r0:], x["v_tail"][:, :, r0:],
-                                              x["k_pre"], x["v_pre"], st.idx, scale, out=out[:, :, :st.idx.numel()],
-                                              status=status, seq_list=st.active_seq, n_seq=B, n_seq_dev=st.active_cnt)
-                                  for x in layers]
-            for pl in plans[key]:
-                pl.launch()
-            return pool[(st.n + st.t) % len(pool)]
-        return forward
-
     res = {"what": "whole block-wise decode (refresh + pruned iterations per block, early exit off); not part of `value`",
-           "workload": cfg.name, "blocks": n_blocks, "B": B, "K": K, "n_layers": cfg.n_layers, "runs": {}}
-    for la in lookaheads:
-        dec = BlockDecoder(B, L, K, cfg.V, tau0=cfg.tau0, alpha=cfg.alpha, mask_id=cfg.V - 1, w_tokens=cfg.w,
-                           keep_last=cfg.keep_last, device=device, lookahead=la)
-        forward = forward_for(dec)
-        dec.decode(forward)                       # warm-up (and the plans)
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n0 = ds.ds_launch_count()
-        a.record()
-        got = dec.decode(forward)
-        b.record()
-        torch.cuda.synchronize()
-        ms = a.elapsed_time(b)
-        res["runs"][f"lookahead{la}"] = {"ms": ms, "iterations": int(sum(got["steps"])),
-                                         "iterations_enqueued": int(sum(got["launched"])),
-                                         "ms_per_iteration": ms / max(1, sum(got["steps"])),
-                                         "launches": int(ds.ds_launch_count() - n0)}
+           "blocks": n_blocks, "K": base.K, "n_layers": base.n_layers, "P": base.P, "batches": {}}
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    for nb in batches:
+        cfg = wl.shrink(base, B=nb, gen=n_blocks * base.K, name=f"llada{nb}x32-decode")
+        B, K, L, P, D = cfg.B, cfg.K, cfg.gen, cfg.P, cfg.D
+        layers = [wl.attention_inputs(cfg, device=device, layer=l) for l in range(cfg.n_layers)]
+        pool = [wl.logits(cfg, device=device, step=s, spike_range=(14.0, 26.0)) for s in range(4)]
+        scale = 1.0 / math.sqrt(D)
+        Lq_max = len(ds.retained_indices(L, K, 0, cfg.w, cfg.keep_last))
+        # refresh iteration: queries and keys are all of prefix + retained rows (one seeded set shared by the layers)
+        dense = wl.attention_inputs(wl.shrink(cfg, P=0, gen=P + Lq_max, name="refresh"), device=device, layer=99)
+        out = torch.empty((B, cfg.Hq, P + Lq_max, D), dtype=cfg.torch_dtype(), device=device)
+        ar = torch.arange(P + Lq_max, dtype=torch.int32, device=device)
+
+        def forward_for(dec):
+            # the calls of a block repeat with the same pointers: plan them once per block
+            plans = {}
+
+            def forward(st):
+                key = (st.n, st.refresh)
+                if key not in plans:
+                    if st.refresh:
+                        n_rows = P + len(ds.retained_indices(L, K, st.n, cfg.w, cfg.keep_last))
+                        one = ds.AttnPlan(dense["q_tail"], dense["k_tail"], dense["v_tail"], None, None, ar[:n_rows],
+                                          scale, out=out[:, :, :n_rows], status=status, seq_list=st.active_seq, n_seq=B,
+                                          n_seq_dev=st.active_cnt)
+                        plans[key] = [one] * cfg.n_layers
+                    else:
+                        r0 = st.n * K
+                        plans[key] = [ds.AttnPlan(x["q_tail"][:, :, r0:], x["k_tail"][:, :, r0:], x["v_tail"][:, :, r0:],
+                                                  x["k_pre"], x["v_pre"], st.idx, scale, out=out[:, :, :st.idx.numel()],
+                                                  status=status, seq_list=st.active_seq, n_seq=B,
+                                                  n_seq_dev=st.active_cnt) for x in layers]
+                for pl in plans[key]:
+                    pl.launch()
+            return forward
+
+        runs = {}
+        for name, la, graphs in (("sync", 0, False), ("lookahead2", 2, False), ("lookahead2_graphs", 2, True)):
+            dec = BlockDecoder(B, L, K, cfg.V, tau0=cfg.tau0, alpha=cfg.alpha, mask_id=cfg.V - 1, w_tokens=cfg.w,
+                               keep_last=cfg.keep_last, device=device, lookahead=la)
+            forward = forward_for(dec)
+            stage = lambda n, t: dec.logits.copy_(pool[(n + t) % len(pool)])
+            dec.decode(forward, before_iteration=stage, graphs=graphs)      # warm-up: plans, graph capture
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n0 = ds.ds_launch_count()
+            a.record()
+            got = dec.decode(forward, before_iteration=stage, graphs=graphs)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b)
+            runs[name] = {"ms": ms, "iterations": int(sum(got["steps"])),
+                          "iterations_enqueued": int(sum(got["launched"])),
+                          "ms_per_iteration": ms / max(1, sum(got["steps"])),
+                          "host_launch_calls": int(ds.ds_launch_count() - n0)}
+            del dec, forward
+        res["batches"][f"B{nb}"] = runs
+        del layers, pool, dense, out
+        torch.cuda.empty_cache()
     res["device_status"] = int(ds.ds_read_status(status))
     return res
 

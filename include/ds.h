@@ -378,6 +378,10 @@ DS_API int ds_block_begin(const ds_block_params *p, void *stream);
 DS_API int ds_read_status(const uint32_t *device_status, void *stream, uint32_t *host_out);
 /* HOST: static string for a ds_status value. */
 DS_API const char *ds_strerror(int code);
+/* The CUDA runtime's error code (cudaError_t as int) and its name for the most recent call on this host
+ * thread that returned DS_ERR_CUDA; 0 / "cudaSuccess" if there was none. */
+DS_API int ds_last_cuda_error(void);
+DS_API const char *ds_last_cuda_error_name(void);
 /* HOST: library version, major * 1000 + minor. */
 DS_API int ds_version(void);
 /* HOST: number of kernels this library has launched in this process (all entry points). */

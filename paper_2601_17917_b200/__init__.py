@@ -36,7 +36,10 @@ _lib = None
 class DsError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {ds_strerror(code)} (status {code})")
+        detail = ""
+        if code == DS_ERR_CUDA:
+            detail = f" [{lib().ds_last_cuda_error_name().decode()} = {lib().ds_last_cuda_error()}]"
+        super().__init__(f"{where}: {ds_strerror(code)} (status {code}){detail}")
 
 
 class _AttnParams(ctypes.Structure):
@@ -136,6 +139,8 @@ def lib() -> ctypes.CDLL:
         L.ds_unmask_select.argtypes = [ctypes.POINTER(_SelectParams), ctypes.c_void_p]
         L.ds_read_status.restype = ctypes.c_int
         L.ds_read_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
+        L.ds_last_cuda_error.restype = ctypes.c_int
+        L.ds_last_cuda_error_name.restype = ctypes.c_char_p
         L.ds_strerror.restype = ctypes.c_char_p
         L.ds_strerror.argtypes = [ctypes.c_int]
         L.ds_version.restype = ctypes.c_int

@@ -11,6 +11,8 @@ namespace ds {
 
 static std::atomic<long long> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+thread_local int g_last_cuda_error = 0;
+void note_cuda_error(int code) { g_last_cuda_error = code; }
 
 int sm_count() {
   static int cached[64];
@@ -264,6 +266,11 @@ int ds_block_begin(const ds_block_params *p, void *stream) {
   if ((long long)p->B * p->K > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   if (p->B > 0 && (!p->eos_exit || !p->masked || !p->x_block || !p->active_seq)) return DS_ERR_INVALID_ARG;
   return ds::launch_block_begin(*p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int ds_last_cuda_error(void) { return ds::g_last_cuda_error; }
+const char *ds_last_cuda_error_name(void) {
+  return cudaGetErrorName(static_cast<cudaError_t>(ds::g_last_cuda_error));
 }
 
 int ds_read_status(const uint32_t *device_status, void *stream, uint32_t *host_out) {

@@ -304,12 +304,11 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           }
           DS_TR(0, issued >> 1, kv * 3 + 1);
           if (j < n_pre) {
-            if (lane == 0) {
+            {
+              // one lane per 64-column chunk: the copies are issued side by side
               const CUtensorMap *map = kv ? &prm.vpre : &prm.kpre;
-#pragma unroll
-              for (int c = 0; c < G_::kChunks; ++c)
-                tma_load_4d(dst + c * kChunkBytes, map, full, c * 64, j * kBlockN, it.hk, it.b);
-              mbar_arrive_expect_tx(full, G_::kTileBytes);
+              if (lane < G_::kChunks) tma_load_4d(dst + lane * kChunkBytes, map, full, lane * 64, j * kBlockN, it.hk, it.b);
+              if (lane == 0) mbar_arrive_expect_tx(full, G_::kTileBytes);
             }
           } else {
             const int t0 = (j - n_pre) * kBlockN;

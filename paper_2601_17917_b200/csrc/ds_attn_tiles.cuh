@@ -56,7 +56,7 @@ __device__ __forceinline__ bool bad_sequence_numbers(const AttnCommon &c, int n_
 // ------------------------------------------------------------------------------------------------
 // Producer helper: fetch n gathered rows (logical rows R0 .. R0+n-1 of a stacked sequence whose
 // period is Lq) into a swizzled tile whose 64-column chunks are chunk_stride bytes apart.  The whole
-// warp calls it; lane 0 issues the copies.  Returns the bytes issued (valid on lane 0).
+// warp calls it; lane 0 issues the copies (a whole-tile fetch: one lane per chunk).  Returns the bytes issued.
 // ------------------------------------------------------------------------------------------------
 template <int D>
 __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUtensorMap *map32, const CUtensorMap *map1,
@@ -70,6 +70,24 @@ __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUt
   if (pos0 >= Lq) {
     head += pos0 / Lq;
     pos0 %= Lq;
+  }
+  // A full tile of consecutive rows inside one head (the current block and its window, every tile of a
+  // cache-refresh step) needs no staging: the list is strictly ascending, so its first and last entry
+  // decide, and one box per 64-column chunk fetches it, each chunk issued by a lane of its own.
+  if (n == 128 && pos0 + 128 <= Lq) {
+    int first, last;
+    if (idx_cache != nullptr && pos0 + 127 < kIdxCap) {
+      first = idx_cache[pos0];
+      last = idx_cache[pos0 + 127];
+    } else {
+      const int32_t *ix = prm.idx + (long long)b * prm.idx_bstride;
+      first = ix[pos0];
+      last = ix[pos0 + 127];
+    }
+    if (last - first == 127 && first >= 0 && last < prm.T) {
+      if (lane < (D / 64)) tma_load_4d(dst + lane * chunk_stride, map128, bar, lane * 64, first, head, b);
+      return 128u * 128u * (D / 64);
+    }
   }
   __syncwarp();
   if (!staged) {  // otherwise idx_s already holds these rows (the K tile of the same rows came first)
@@ -93,14 +111,6 @@ __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUt
   }
   uint32_t bytes = 0;
   if (lane == 0) {
-    // a full tile of consecutive rows inside one head (the current block and its window, every tile of a
-    // cache-refresh step): one box per 64-column chunk.  The list is strictly ascending, so first and last
-    // entry decide.
-    if (n == 128 && pos0 + 128 <= Lq && idx_s[127] - idx_s[0] == 127) {
-#pragma unroll
-      for (int c = 0; c < (D / 64); ++c) tma_load_4d(dst + c * chunk_stride, map128, bar, c * 64, idx_s[0], head, b);
-      return 128u * 128u * (D / 64);
-    }
     int r = 0, pos = pos0;
     while (r < n) {
       const int row = idx_s[r];

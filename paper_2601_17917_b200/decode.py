@@ -80,15 +80,62 @@ class BlockDecoder:
         # slot j of a block: number of active sequences before iteration j, copied to pinned memory
         self.cnt_host = torch.zeros(K + 1, dtype=torch.int32).pin_memory()
         self.events = [torch.cuda.Event() for _ in range(K + 1)]
+        self._graphs = {}
 
     def _publish(self, slot: int, cnt: torch.Tensor):
         self.cnt_host[slot:slot + 1].copy_(cnt, non_blocking=True)
         self.events[slot].record()
 
-    def decode(self, forward) -> dict:
+    def _iteration(self, forward, n: int, t: int):
+        """One iteration of block n: the model callback, Eq. 4 at the rows still masked, the selection."""
+        B, K = self.B, self.K
+        z = forward(Step(n=n, t=t, refresh=(t == 0), idx=self.idx_all[n] if t == 0 else self.idx[n],
+                         active_seq=self.active, active_cnt=self.active_cnt, x_block=self.x_block,
+                         logits=self.logits))
+        if z is None:
+            z = self.logits
+        elif z.shape != self.logits.shape or z.dtype != self.logits.dtype or z.device != self.logits.device:
+            raise ValueError("forward returned logits of the wrong shape, type or device")
+        ds_confidence_listed(z, self.masked_rows, self.masked_cnt, self.conf, self.tok,
+                             n_listed_max=B * K, workspace=self.workspace)
+        ds_unmask_select(self.conf.view(B, K), self.tok.view(B, K), self.masked, self.x_block, self.tau0,
+                         self.alpha, ratio_extra=self.extra[n], eos_id=self.eos_id, eos_tau=self.eos_tau,
+                         seq_list=self.active, n_seq=B, n_seq_dev=self.active_cnt, out=self.sel)
+
+    def _graph(self, forward, n: int, refresh: bool):
+        """The CUDA graph of an iteration of block n (one for the refresh iteration, one for all the others:
+        nothing an iteration is launched with depends on t).  Before the first capture every kernel runs once
+        on empty lists, so that no module is loaded while a capture is open."""
+        key = (n, refresh)
+        if key not in self._graphs:
+            t = 0 if refresh else 1
+            self.active_cnt.zero_()
+            self.masked_cnt.zero_()
+            self._iteration(forward, n, t)          # empty lists: launches everything, changes nothing
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self._iteration(forward, n, t)
+            self._graphs[key] = g
+        return self._graphs[key]
+
+    def capture(self, forward):
+        """Captures the graphs of every block ahead of a ``decode(..., graphs=True)`` (which otherwise captures
+        them on first use).  ``forward`` must be the callable later passed to ``decode``: it has to launch the
+        same work on the same buffers whenever it is called for a given (block, refresh) and must not depend
+        on the iteration number, allocate, or synchronise."""
+        for n in range(self.N):
+            self._graph(forward, n, True)
+            self._graph(forward, n, False)
+
+    def decode(self, forward, before_iteration=None, graphs: bool = False) -> dict:
         """Runs the whole procedure on the current stream.  Returns x [B, L] (device), steps [N] (iterations
-        each block needed), launched [N] (iterations enqueued, >= steps) and eos_exit [B] (device)."""
+        each block needed), launched [N] (iterations enqueued, >= steps) and eos_exit [B] (device).
+        ``before_iteration(n, t)``, if given, runs eagerly ahead of every iteration (e.g. to stage inputs).
+        With ``graphs`` an iteration is one CUDA-graph launch (see ``capture``)."""
         B, K, N = self.B, self.K, self.N
+        if graphs:
+            self.capture(forward)
         self.x.fill_(self.mask_id)
         self.eos_exit.zero_()
         steps, launched = [], []
@@ -103,18 +150,12 @@ class BlockDecoder:
                     self.events[seen].synchronize()
                     if int(self.cnt_host[seen]) == 0:
                         break
-                z = forward(Step(n=n, t=t, refresh=(t == 0), idx=self.idx_all[n] if t == 0 else self.idx[n],
-                                 active_seq=self.active, active_cnt=self.active_cnt, x_block=self.x_block,
-                                 logits=self.logits))
-                if z is None:
-                    z = self.logits
-                elif z.shape != self.logits.shape or z.dtype != self.logits.dtype or z.device != self.logits.device:
-                    raise ValueError("forward returned logits of the wrong shape, type or device")
-                ds_confidence_listed(z, self.masked_rows, self.masked_cnt, self.conf, self.tok,
-                                     n_listed_max=B * K, workspace=self.workspace)
-                ds_unmask_select(self.conf.view(B, K), self.tok.view(B, K), self.masked, self.x_block, self.tau0,
-                                 self.alpha, ratio_extra=self.extra[n], eos_id=self.eos_id, eos_tau=self.eos_tau,
-                                 seq_list=self.active, n_seq=B, n_seq_dev=self.active_cnt, out=self.sel)
+                if before_iteration is not None:
+                    before_iteration(n, t)
+                if graphs:
+                    self._graphs[(n, t == 0)].replay()
+                else:
+                    self._iteration(forward, n, t)
                 t += 1
                 self._publish(t, self.active_cnt)
             self.events[t].synchronize()             # everything enqueued for this block has run

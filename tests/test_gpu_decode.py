@@ -121,6 +121,23 @@ def test_every_sequence_exits_and_the_last_blocks_take_no_iteration():
         assert np.array_equal(got["x"].cpu().numpy(), ref["x"])
 
 
+def test_iterations_as_cuda_graphs():
+    # one graph launch per iteration; the logits are staged by the eager hook, the captured callback is fixed
+    cfg = _cfg(4, 16, 64, 512, seed=11)
+    B, K, L, V = cfg.B, cfg.K, cfg.gen, cfg.V
+    z = _table(cfg)
+    ref = oracle.decode(lambda n, t: z(n, t).float().numpy().reshape(B, K, V), B, L, K, cfg.tau0, 0.3, MASK)
+    dec = BlockDecoder(B, L, K, V, tau0=cfg.tau0, alpha=0.3, mask_id=MASK, w_tokens=16, device=DEV, lookahead=2)
+    stage = lambda n, t: dec.logits.copy_(z(n, t).to(DEV))
+    n0 = ds.ds_launch_count()
+    for _ in range(2):                                  # the second run replays the graphs captured by the first
+        got = dec.decode(lambda st: None, before_iteration=stage, graphs=True)
+        torch.cuda.synchronize()
+        assert np.array_equal(got["x"].cpu().numpy(), ref["x"])
+        assert got["steps"] == ref["steps"].tolist()
+    assert len(dec._graphs) == 2 * (L // K)
+
+
 def test_block_begin_lists():
     B, K = 70, 24
     rng = np.random.default_rng(3)
