@@ -195,6 +195,7 @@ class Step:
         x0, m0 = wl.block_state(cfg, "all")
         self.x0, self.m0 = x0.to(device), m0.to(device)
         self.x_block, self.masked = self.x0.clone(), self.m0.clone()
+        self.no_exit = torch.zeros(cfg.B, dtype=torch.uint8, device=device)
         dt = cfg.torch_dtype()
         B, K = cfg.B, cfg.K
         self.out = torch.empty((B, cfg.Hq, self.Lq, cfg.D), dtype=dt, device=device)
@@ -224,9 +225,9 @@ class Step:
 
     def select(self):
         cfg = self.cfg
-        # every timed step starts from the same block state (two small device-to-device copies)
-        self.masked.copy_(self.m0)
-        self.x_block.copy_(self.x0)
+        # every timed step starts from the state a block begins with (every position masked)
+        self.ds.ds_block_begin(self.no_exit, self.masked, self.x_block, cfg.V - 1, cfg.V - 2, self.sel["active_seq"],
+                               self.sel["active_cnt"])
         self.ds.ds_unmask_select(self.conf.view(cfg.B, cfg.K), self.tok.view(cfg.B, cfg.K), self.masked, self.x_block,
                                  cfg.tau0, cfg.alpha, eos_id=cfg.V - 2, eos_tau=cfg.tau0, out=self.sel)
 
