@@ -87,6 +87,25 @@ size_t ds_attn_pruned_workspace(const ds_attn_params *p) {
 
 namespace ds {
 namespace {
+// Several M-tiles per KV head (wide windows, the unpruned reference, a cache-refresh step): the two-tile
+// kernel fetches every KV tile once for a pair of M-tiles and keeps the softmax warps busy on one tile while
+// the tensor pipe works for the other.  Measured per work item it costs about 1.8 single tiles for a full pair
+// and 1.6 for a lone tile (no second S buffer to run ahead with), so it pays when the pairs are mostly full
+// and the number of rounds over the SMs does not grow.
+bool two_tile_kernel_pays(const ds_attn_params &p) {
+  const long long rows = (long long)(p.Hq / p.Hkv) * p.Lq;
+  const long long n_full = rows / 128, rem = rows % 128;
+  // the one-tile kernel serves a remainder of up to 8 rows together with the last full tile
+  const long long n_mt1 = (p.D == 128 && n_full >= 1 && rem >= 1 && rem <= 8) ? n_full : n_full + (rem ? 1 : 0);
+  const long long n_mt = n_full + (rem ? 1 : 0), n_pr = (n_mt + 1) / 2;
+  if (n_mt < 2) return false;
+  const long long heads = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv, sms = sm_count();
+  const double rounds1 = (double)((heads * n_mt1 + sms - 1) / sms);
+  const double rounds2 = (double)((heads * n_pr + sms - 1) / sms);
+  const double pair_cost = (1.8 * (double)(n_mt / 2) + 1.6 * (double)(n_mt % 2)) / (double)n_pr;
+  return rounds2 * pair_cost < 0.97 * rounds1;
+}
+
 // Validation, choice of the kernel and its parameters for one set of arguments.
 int resolve_attn(const ds_attn_params *p, AttnPrepared &a) {
   const int rc = validate_attn(p);
@@ -102,9 +121,7 @@ int resolve_attn(const ds_attn_params *p, AttnPrepared &a) {
   if (tc_ok && path != AttnPath::kSimt) {
     const size_t need = attn_tc_workspace_bytes(*p);
     if (need > 0 && (!p->workspace || !aligned(p->workspace, 256) || p->workspace_bytes < need)) return DS_ERR_WORKSPACE;
-    // The two-tile kernel (one KV tile shared by two M-tiles) stays selectable through DS_ATTN_PATH=tc2 but is
-    // not dispatched: once consecutive retained rows are fetched as whole-tile boxes the one-tile kernel is
-    // the faster one on every measured shape, pruned or dense.
+    if (path == AttnPath::kAuto && two_tile_kernel_pays(*p)) return prepare_attn_tc2(*p, a);
     return prepare_attn_tc(*p, a);
   }
   a.grid = 1;  // the SIMT launcher sizes its own grid from a.p

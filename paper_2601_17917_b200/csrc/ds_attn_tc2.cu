@@ -1,15 +1,16 @@
 // ds_attn_pruned, tensor-core path for bf16 when the stacked query rows of a KV head fill more than one
-// 128-row M-tile (GQA groups, wide windows, the unpruned reference): there the problem is bound by the
-// tensor cores and the exponential unit, not by the KV stream, and the shape of the kernel follows.
+// 128-row M-tile (GQA groups, wide windows, the unpruned reference, a cache-refresh step): there the
+// problem is bound by the tensor cores and the softmax, not by the KV stream, and the shape of the kernel
+// follows.
 //
 // Work item = (batch, KV head, PAIR of 128-row M-tiles).  Both tiles of a pair use every KV tile once
-// from shared memory (half the shared-memory and L2 traffic per MMA of the one-tile kernel), and their
-// softmax runs on two warpgroups that alternate with the tensor pipe: while warpgroup A exponentiates
-// S_a of KV tile j, the pipe runs P_b V and Q_b K^T; then the roles swap.
+// from shared memory (half the shared-memory and L2 traffic per MMA of the one-tile kernel), and the
+// softmax warps alternate with the tensor pipe: while they exponentiate S_a of KV tile j, the pipe runs
+// P_b V and Q_b K^T; then the roles swap.
 //
 // Warp roles (320 threads, one CTA per SM):
-//   warps 0-3  softmax + epilogue of M-tile a (thread = row, 128 columns in registers)
-//   warps 4-7  the same for M-tile b (idle when the pair has only one tile)
+//   warps 0-7  softmax + epilogue, M-tile a then M-tile b of every KV tile: half a row (64 columns) per
+//              thread, the two halves of a row in the two half-warps (16x32bx2 TMEM accesses)
 //   warp  8    TMA producer (prefix tiles by tiled boxes, tail rows gathered through the index list)
 //   warp  9    TMEM allocation, MMA issue (one elected lane), in the order
 //              P_a V(j-1), Q_a K(j)^T, P_b V(j-1), Q_b K(j)^T
@@ -109,11 +110,11 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
     mbar_init(bar_q_free, 1);
     mbar_init(bar_s_full, 1);
     mbar_init(bar_s_full + 8, 1);
-    mbar_init(bar_p_full, 4);
-    mbar_init(bar_p_full + 8, 4);
+    mbar_init(bar_p_full, 8);
+    mbar_init(bar_p_full + 8, 8);
     mbar_init(bar_o_full, 1);
-    mbar_init(bar_o_free, 4);
-    mbar_init(bar_o_free + 8, 4);
+    mbar_init(bar_o_free, 8);
+    mbar_init(bar_o_free + 8, 8);
     for (int s = 0; s < G_::kSlots; ++s) {
       mbar_init(bar_slot_full + 8 * s, 1);
       mbar_init(bar_slot_empty + 8 * s, 1);
@@ -336,137 +337,145 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
     }
     timed_out = !ok;
   } else {
-    // ============================ softmax + epilogue (warpgroup x = warp / 4 owns M-tile x) ============================
-    const int x = warp >> 2;
-    const int row = (warp & 3) * 32 + lane;  // TMEM lane = row of the M-tile
-    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t s_base = lane_base + G_::kTmemS + 128 * x, o_base = lane_base + G_::kTmemO + 128 * x;
+    // ============================ softmax + epilogue ============================
+    // All eight warps take M-tile a, then M-tile b, of every KV tile: half a row (64 columns) per thread, the
+    // two halves of a row in the two half-warps (16x32bx2 accesses).  While they work on one M-tile the
+    // issuer runs P V and the next Q K^T of the other.
+    const int half = lane >> 4;                            // column half this thread works on
+    const int lane0 = (warp & 3) * 32 + (warp >> 2) * 16;   // first TMEM lane of this warp
+    const int row = lane0 + (lane & 15);                   // TMEM lane = row of the M-tile
+    const uint32_t lane_base = tmem + ((uint32_t)lane0 << 16);
     const float c2 = prm.scale_log2;
+    constexpr int kOCols = D / 2;                          // accumulator columns per thread
     bool ok = true;
-    int g0 = 0, k = 0;  // g0: tiles this warpgroup's M-tile has seen before the current item
+    int ga0 = 0, gb0 = 0, k = 0;  // tiles M-tile a / b have seen before the current item (phase counts of their barriers)
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k) {
       const Item2 it = decode_item2(prm, item);
-      const int my_rows = x ? it.rows_b : it.rows_a;
-      if (my_rows == 0) {
-        // no tile for this warpgroup in this item: stay in step with the per-item barriers only
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full, k & 1, abort_flag));
-        if (!ok) break;
-        if (lane == 0) mbar_arrive(bar_o_free + 8 * x);
-        continue;
-      }
-      const bool live = row < my_rows;
-      float m_used = -INFINITY, l_sum = 0.f;
-      for (int j = 0; j < n_tiles; ++j) {
-        const int g = g0 + j;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * x, g & 1, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t s[128];
-        tmem_ld32(s_base, &s[0]);
-        tmem_ld32(s_base + 32, &s[32]);
-        tmem_ld32(s_base + 64, &s[64]);
-        tmem_ld32(s_base + 96, &s[96]);
-        tmem_wait_ld();
+      const int n_x = it.rows_b > 0 ? 2 : 1;
+      float m_used[2] = {-INFINITY, -INFINITY};  // maximum the probabilities are expressed against (log2 units)
+      float l_sum[2] = {0.f, 0.f};               // this thread's half of the row sum
+      for (int j = 0; j < n_tiles && ok; ++j) {
         const int valid = (j < n_pre) ? min(kBlockN, prm.P - j * kBlockN) : min(kBlockN, prm.Lq - (j - n_pre) * kBlockN);
-        if (valid < kBlockN) {
 #pragma unroll
-          for (int c = 0; c < 128; ++c)
-            if (c >= valid) s[c] = 0xff800000u;  // -inf
-        }
-        float mx;
-        {
-          float a[8];
+        for (int x = 0; x < 2; ++x) {
+          if (x >= n_x) break;
+          const bool live = row < (x ? it.rows_b : it.rows_a);
+          const int gx = (x ? gb0 : ga0) + j;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * x, gx & 1, abort_flag));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t s_base = lane_base + G_::kTmemS + 128 * x, o_base = lane_base + G_::kTmemO + 128 * x;
+          uint32_t s[64];
+          tmem_ld16x2_32<64>(s_base, &s[0]);        // columns 64 half + 0..31
+          tmem_ld16x2_32<64>(s_base + 32, &s[32]);  // columns 64 half + 32..63
+          tmem_wait_ld();
+          if (valid < kBlockN) {
 #pragma unroll
-          for (int c = 0; c < 8; ++c) a[c] = __uint_as_float(s[c]);
-#pragma unroll
-          for (int c = 8; c < 120; c += 16) {
-#pragma unroll
-            for (int u = 0; u < 8; ++u) a[u] = fmax3(a[u], __uint_as_float(s[c + u]), __uint_as_float(s[c + 8 + u]));
+            for (int c = 0; c < 64; ++c)
+              if (c + 64 * half >= valid) s[c] = 0xff800000u;  // -inf: columns past the end of a partial tile
           }
+          float mx;
+          {
+            float a[8];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) a[u] = fmaxf(a[u], __uint_as_float(s[120 + u]));
-          mx = fmaxf(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]));
-          mx = fmax3(mx, a[6], a[7]);
-        }
-        const float m_tile = mx * c2;
-        float factor = 1.f;
-        if (m_tile > m_used + kRescaleThreshold || m_used == -INFINITY) {
-          factor = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_tile);
-          m_used = m_tile;
-        }
-        const bool warp_rescales = __any_sync(0xffffffffu, live && factor != 1.f) && (j > 0);
-        l_sum *= factor;
-        if (warp_rescales) {
-          // S of this tile being complete means every MMA issued before its Q K^T has completed, the
-          // previous P V among them: O_x is quiescent
+            for (int c = 0; c < 8; ++c) a[c] = __uint_as_float(s[c]);
 #pragma unroll
-          for (int cb = 0; cb < D; cb += 32) {
-            uint32_t o[32];
-            tmem_ld32(o_base + cb, o);
-            tmem_wait_ld();
+            for (int c = 8; c < 56; c += 16) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor);
-            tmem_st32(o_base + cb, o);
+              for (int u = 0; u < 8; ++u) a[u] = fmax3(a[u], __uint_as_float(s[c + u]), __uint_as_float(s[c + 8 + u]));
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) a[u] = fmaxf(a[u], __uint_as_float(s[56 + u]));
+            mx = fmaxf(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]));
+            mx = fmax3(mx, a[6], a[7]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
           }
-        }
-        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-        const float neg_m = -m_used;
+          const float m_tile = mx * c2;
+          float factor = 1.f;
+          if (m_tile > m_used[x] + kRescaleThreshold || m_used[x] == -INFINITY) {
+            factor = (m_used[x] == -INFINITY) ? 0.f : ex2_approx(m_used[x] - m_tile);
+            m_used[x] = m_tile;
+          }
+          const bool warp_rescales = __any_sync(0xffffffffu, live && factor != 1.f) && (j > 0);
+          l_sum[x] *= factor;
+          if (warp_rescales) {
+            // S of this tile being complete means every MMA issued before its Q K^T has completed, the
+            // previous P V of this M-tile among them: O_x is quiescent
 #pragma unroll
-        for (int c = 0; c < 64; c += 2) {
-          const float p0 = ex2_approx(fmaf(__uint_as_float(s[2 * c]), c2, neg_m));
-          const float p1 = ex2_approx(fmaf(__uint_as_float(s[2 * c + 1]), c2, neg_m));
-          const float p2 = ex2_approx(fmaf(__uint_as_float(s[2 * c + 2]), c2, neg_m));
-          const float p3 = ex2_approx(fmaf(__uint_as_float(s[2 * c + 3]), c2, neg_m));
-          s[c] = pack_bf16(p0, p1);  // P overwrites the registers of the S values it no longer needs
-          s[c + 1] = pack_bf16(p2, p3);
-          l0 += p0;
-          l1 += p1;
-          l2 += p2;
-          l3 += p3;
+            for (int cb = 0; cb < kOCols; cb += 32) {
+              uint32_t o[32];
+              tmem_ld16x2_32<kOCols>(o_base + cb, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor);
+              tmem_st16x2_32<kOCols>(o_base + cb, o);
+            }
+          }
+          float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+          const float neg_m = -m_used[x];
+          uint32_t pk[32];
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(s[2 * c]), c2, neg_m));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(s[2 * c + 1]), c2, neg_m));
+            const float p2 = ex2_approx(fmaf(__uint_as_float(s[2 * c + 2]), c2, neg_m));
+            const float p3 = ex2_approx(fmaf(__uint_as_float(s[2 * c + 3]), c2, neg_m));
+            pk[c] = pack_bf16(p0, p1);
+            pk[c + 1] = pack_bf16(p2, p3);
+            l0 += p0;
+            l1 += p1;
+            l2 += p2;
+            l3 += p3;
+          }
+          l_sum[x] += (l0 + l1) + (l2 + l3);
+          // P row -> TMEM over the first 64 columns of S_x (two bf16 per column); this thread's 64 keys are
+          // columns 32 half .. 32 half + 31
+          tmem_st16x2_32<32>(s_base, pk);
+          tmem_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_p_full + 8 * x);
         }
-        l_sum += (l0 + l1) + (l2 + l3);
-        // P row -> TMEM over the first 64 columns of S_x (two bf16 per column)
-        tmem_st32(s_base, &s[0]);
-        tmem_st32(s_base + 32, &s[32]);
-        tmem_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_p_full + 8 * x);
       }
       if (!ok) break;
+      // ---- epilogue of the item: the last P V of both M-tiles has completed ----
       ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full, k & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
-      const int R = (it.pr * 2 + x) * kBlockM + row;
-      const int hq = it.hk * prm.G + (live ? R / prm.Lq : 0), i = live ? R % prm.Lq : 0;
-      const float inv = 1.f / l_sum;
-      __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(prm.out) + it.b * prm.out_stride[0] + hq * prm.out_stride[1] +
-                            (long long)i * prm.out_stride[2];
 #pragma unroll
-      for (int cb = 0; cb < D; cb += 32) {
-        uint32_t o[32];
-        tmem_ld32(o_base + cb, o);
-        tmem_wait_ld();
-        if (cb + 32 >= D) {
-          // everything of O_x is in registers or stored: the next item may overwrite it
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_o_free + 8 * x);
+      for (int x = 0; x < 2; ++x) {
+        const bool have = x < n_x;
+        const bool live = have && row < (x ? it.rows_b : it.rows_a);
+        uint32_t o[kOCols];
+        if (have) {
+#pragma unroll
+          for (int cb = 0; cb < kOCols; cb += 32) tmem_ld16x2_32<kOCols>(lane_base + G_::kTmemO + 128 * x + cb, &o[cb]);
+          tmem_wait_ld();
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_o_free + 8 * x);   // O_x is in registers (or does not exist): it may be overwritten
+        const float l_row = l_sum[x] + __shfl_xor_sync(0xffffffffu, l_sum[x], 16);  // the other half of the row
         if (live) {
+          const int R = (it.pr * 2 + x) * kBlockM + row;
+          const int hq = it.hk * prm.G + R / prm.Lq, i = R % prm.Lq;
+          const float inv = 1.f / l_row;
+          __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(prm.out) + it.b * prm.out_stride[0] +
+                                hq * prm.out_stride[1] + (long long)i * prm.out_stride[2] + kOCols * half;
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
+          for (int c = 0; c < kOCols; c += 8) {
             uint4 w;
-            w.x = pack_bf16(__uint_as_float(o[8 * q + 0]) * inv, __uint_as_float(o[8 * q + 1]) * inv);
-            w.y = pack_bf16(__uint_as_float(o[8 * q + 2]) * inv, __uint_as_float(o[8 * q + 3]) * inv);
-            w.z = pack_bf16(__uint_as_float(o[8 * q + 4]) * inv, __uint_as_float(o[8 * q + 5]) * inv);
-            w.w = pack_bf16(__uint_as_float(o[8 * q + 6]) * inv, __uint_as_float(o[8 * q + 7]) * inv);
-            *reinterpret_cast<uint4 *>(orow + cb + 8 * q) = w;
+            w.x = pack_bf16(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+            *reinterpret_cast<uint4 *>(orow + c) = w;
           }
+          if (prm.lse && half == 0) prm.lse[((long long)it.b * prm.Hq + hq) * prm.Lq + i] = (m_used[x] + log2f(l_row)) * kLn2;
         }
       }
-      if (live && prm.lse) prm.lse[((long long)it.b * prm.Hq + hq) * prm.Lq + i] = (m_used + log2f(l_sum)) * kLn2;
-      g0 += n_tiles;
+      ga0 += n_tiles;
+      if (n_x == 2) gb0 += n_tiles;
     }
     timed_out = !ok;
   }
