@@ -89,8 +89,12 @@ typedef enum { DS_F32 = 0, DS_BF16 = 1 } ds_dtype;
  * Envelope: D in {64, 128} for the tensor-core bf16 path; the fp32 path takes
  * any D that is a multiple of 32 up to 256.  Hq % Hkv == 0.  1 <= Lq <= T.
  *
- * Workspace: ds_attn_pruned_workspace(p) bytes, 256-byte aligned, used for
- * split-KV partial results; contents need not be preserved between calls.
+ * Workspace: ds_attn_pruned_workspace(p) bytes, 256-byte aligned; contents need
+ * not be preserved between calls.  It is used when the call has few work
+ * items (small batches with a long prefix): the keys of every item are then
+ * split over several CTAs, which leave normalised partial results and their
+ * log-sum-exp in the workspace, and a second kernel merges them.  A call
+ * without a (large enough) workspace is not an error; it runs unsplit.
  * Errors: DS_ERR_INVALID_ARG / DS_ERR_UNSUPPORTED / DS_ERR_WORKSPACE before
  * anything is launched; DS_ERR_CUDA if a launch fails.
  * ------------------------------------------------------------------------ */

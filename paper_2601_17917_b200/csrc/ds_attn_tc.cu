@@ -117,14 +117,32 @@ static_assert(Geo<64>::kSmemBytes <= 227 * 1024, "shared memory budget");
 struct TcParams : attn::AttnCommon {
   int n_mtiles;  // M-tiles per (batch, KV head)
   int x_rows;    // extra rows riding with the last M-tile (0 = none)
-  int n_items;   // B * Hkv * n_mtiles
+  int n_items;   // B * Hkv * n_mtiles * splits
+  // Few work items (small batches): the KV tiles of an item are split over `splits` CTAs, each writing a
+  // normalised partial result and its log-sum-exp to the workspace (out / lse then point there, one copy per
+  // split, split_stride elements apart); a second kernel merges them.
+  int splits, tiles_per_split, n_tiles;
+  long long out_split_stride, lse_split_stride;
 };
 
 struct Item {
   int b, hk, mt, m_rows, x_rows;
+  int split, t0, nt;  // this CTA's KV tiles: t0 .. t0 + nt - 1 of the item's sequence of tiles
 };
+// kSplit = false is the launch in which every item takes all its KV tiles: nothing of the split arithmetic
+// is left in that instantiation.
+template <bool kSplit>
 __device__ __forceinline__ Item decode_item(const TcParams &prm, int item) {
   Item it;
+  it.split = 0;
+  it.t0 = 0;
+  it.nt = prm.n_tiles;
+  if constexpr (kSplit) {
+    it.split = item % prm.splits;
+    item /= prm.splits;
+    it.t0 = it.split * prm.tiles_per_split;
+    it.nt = min(prm.tiles_per_split, prm.n_tiles - it.t0);
+  }
   it.mt = item % prm.n_mtiles;
   const int bh = item / prm.n_mtiles;
   it.hk = bh % prm.Hkv;
@@ -138,7 +156,7 @@ __device__ __forceinline__ Item decode_item(const TcParams &prm, int item) {
 // ------------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------------
-template <int D>
+template <int D, bool kSplit>
 __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_constant__ TcParams prm) {
   using G_ = Geo<D>;
   extern __shared__ uint8_t smem_raw[];
@@ -206,7 +224,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
   const uint32_t tmem = *tmem_base_s;
   // sequences (hence work items) of this launch: all, or the listed ones with the count read on the device
   const int n_live = attn::live_sequences(prm);
-  const int n_items = n_live * prm.Hkv * prm.n_mtiles;
+  const int n_items = n_live * prm.Hkv * prm.n_mtiles * (kSplit ? prm.splits : 1);
   bool timed_out = false;
 
   if (warp == kProducerWarp) {
@@ -250,7 +268,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     // Requests the query tile(s) of this CTA's kq-th item.  The caller has made sure the previous
     // item's last Q K^T has completed.
     auto issue_q = [&](int kq) {
-      const Item it = decode_item(prm, blockIdx.x + kq * gridDim.x);
+      const Item it = decode_item<kSplit>(prm, blockIdx.x + kq * gridDim.x);
       uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
                                       it.mt * kBlockM, it.m_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
       if (it.x_rows > 0) {
@@ -265,8 +283,10 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     };
     int issued = 0;  // ring fills issued so far
     for (int k = 0; k < n_my && !timed_out; ++k) {
-      const Item it = decode_item(prm, blockIdx.x + k * gridDim.x);
-      for (int j = 0; j < n_tiles && !timed_out; ++j) {
+      const Item it = decode_item<kSplit>(prm, blockIdx.x + k * gridDim.x);
+      const int nt_it = kSplit ? it.nt : n_tiles;
+      for (int jj = 0; jj < nt_it && !timed_out; ++jj) {
+        const int j = (kSplit ? it.t0 : 0) + jj;
         for (int kv = 0; kv < 2; ++kv) {
           const int slot = issued % G_::kSlots, use = issued / G_::kSlots;
           const uint32_t dst = sbase + G_::kOffRing + slot * G_::kTileBytes;
@@ -367,11 +387,16 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     int g0 = 0;   // tiles processed by this CTA before the current item
     int k = 0;
     int gx0 = 0;  // tiles of items with extra rows before the current item
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
-      const bool has_x = (D == 128) && decode_item(prm, item).x_rows > 0;
+    int nt_cur = 0;  // KV tiles of the current item that this CTA processes
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += nt_cur) {
+      const int j_lo = kSplit ? decode_item<kSplit>(prm, item).t0 : 0;
+      nt_cur = kSplit ? decode_item<kSplit>(prm, item).nt : n_tiles;
+      const bool has_x = (D == 128) && decode_item<kSplit>(prm, item).x_rows > 0;
       ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full, k & 1, abort_flag));
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int g = g0 + j, gx = gx0 + j;
+      for (int jj = 0; jj < nt_cur && ok; ++jj) {
+        const int j = j_lo + jj;
+        (void)j;
+        const int g = g0 + jj, gx = gx0 + jj;
         const int fill = 2 * g, slot = fill % G_::kSlots, use = fill / G_::kSlots;
         // the K tile has landed, and S[g % 2] is free: P V of tile g - 2, the reader of the P it still
         // holds, has completed
@@ -418,12 +443,12 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
             umma_commit(bar_sx_full + 8 * (gx & 1));
           }
           umma_commit(bar_slot_empty + 8 * slot);
-          if (j == n_tiles - 1) umma_commit(bar_q_free);
+          if (jj == nt_cur - 1) umma_commit(bar_q_free);
           DS_TR(1, g, 1);
         }
         __syncwarp();
       }
-      if (has_x) gx0 += n_tiles;
+      if (has_x) gx0 += nt_cur;
     }
     timed_out = !ok;
   } else if (warp == kPvWarp) {
@@ -437,14 +462,19 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     int g0 = 0, k = 0;
     int kx = 0;   // items with extra rows before the current one
     int gx0 = 0;  // tiles of such items
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
-      const bool has_x = (D == 128) && decode_item(prm, item).x_rows > 0;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int g = g0 + j, gx = gx0 + j;
+    int nt_cur = 0;  // KV tiles of the current item that this CTA processes
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += nt_cur) {
+      const int j_lo = kSplit ? decode_item<kSplit>(prm, item).t0 : 0;
+      nt_cur = kSplit ? decode_item<kSplit>(prm, item).nt : n_tiles;
+      const bool has_x = (D == 128) && decode_item<kSplit>(prm, item).x_rows > 0;
+      for (int jj = 0; jj < nt_cur && ok; ++jj) {
+        const int j = j_lo + jj;
+        (void)j;
+        const int g = g0 + jj, gx = gx0 + jj;
         const int fill = 2 * g + 1, slot = fill % G_::kSlots, use = fill / G_::kSlots;
         bool w = mbar_wait2(bar_slot_full + 8 * slot, use & 1, bar_p_full + 8 * (g & 1), (g >> 1) & 1, abort_flag);
         // the epilogue of the previous item has read O before this item's first P V overwrites it
-        if (j == 0 && k > 0) w = w && mbar_wait(bar_o_free, (k - 1) & 1, abort_flag);
+        if (jj == 0 && k > 0) w = w && mbar_wait(bar_o_free, (k - 1) & 1, abort_flag);
         if (!__all_sync(0xffffffffu, w)) {
           ok = false;
           break;
@@ -456,14 +486,14 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
 #pragma unroll
           for (int ks = 0; ks < kBlockN / 16; ++ks)
             umma_ts(tm + G_::kTmemO, tm + ((g & 1) ? G_::kTmemS1 : G_::kTmemS0) + ks * 8, dv + ((ks * 2048) >> 4),
-                    idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                    idesc_pv, (jj > 0 || ks > 0) ? 1u : 0u);
           umma_commit(bar_pv_done + 8 * (g & 1));  // frees S[g % 2] for Q K^T of tile g + 2
         }
         __syncwarp();
         if (has_x) {
           // the transposed problem's probabilities come from their own warps
           bool wx = mbar_wait(bar_px_full + 8 * (gx & 1), (gx >> 1) & 1, abort_flag);
-          if (j == 0 && kx > 0) wx = wx && mbar_wait(bar_ox_free, (kx - 1) & 1, abort_flag);
+          if (jj == 0 && kx > 0) wx = wx && mbar_wait(bar_ox_free, (kx - 1) & 1, abort_flag);
           if (!__all_sync(0xffffffffu, wx)) {
             ok = false;
             break;
@@ -476,20 +506,20 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
 #pragma unroll
               for (int ks = 0; ks < kBlockN / 16; ++ks) {
                 const uint32_t offx = ((gx & 1) * 2 * kXChunkBytes + (ks / 4) * kXChunkBytes + (ks % 4) * 32) >> 4;
-                umma_ss(tm + G_::kTmemOx, dv + ((ks * 2048) >> 4), dpx + offx, idesc_pv_x, (j > 0 || ks > 0) ? 1u : 0u);
+                umma_ss(tm + G_::kTmemOx, dv + ((ks * 2048) >> 4), dpx + offx, idesc_pv_x, (jj > 0 || ks > 0) ? 1u : 0u);
               }
               umma_commit(bar_pvx_done + 8 * (gx & 1));
             }
           }
           umma_commit(bar_slot_empty + 8 * slot);
-          if (j == n_tiles - 1) umma_commit(bar_o_full);
+          if (jj == nt_cur - 1) umma_commit(bar_o_full);
           DS_TR(1, g, 3);
         }
         __syncwarp();
       }
       if (has_x) {
         ++kx;
-        gx0 += n_tiles;
+        gx0 += nt_cur;
       }
     }
     timed_out = !ok;
@@ -514,8 +544,11 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       ++n_y;
       return __all_sync(0xffffffffu, w);
     };
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
-      const Item it = decode_item(prm, item);
+    int nt_cur = 0;  // KV tiles of the current item that this CTA processes
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += nt_cur) {
+      const int j_lo = kSplit ? decode_item<kSplit>(prm, item).t0 : 0;
+      nt_cur = kSplit ? decode_item<kSplit>(prm, item).nt : n_tiles;
+      const Item it = decode_item<kSplit>(prm, item);
       if (!((D == 128) && it.x_rows > 0)) {
         // nothing to do, but stay in step with the per-item barrier (a parity wait cannot skip phases)
         ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full, k & 1, abort_flag));
@@ -524,8 +557,9 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       float mref[kXMax], lx[kXMax];
 #pragma unroll
       for (int i = 0; i < kXMax; ++i) mref[i] = 0.f, lx[i] = 0.f;
-      for (int j = 0; j < n_tiles; ++j) {
-        const int gx = gx0 + j;
+      for (int jj = 0; jj < nt_cur; ++jj) {
+        const int j = j_lo + jj;
+        const int gx = gx0 + jj;
         // S_x^T of this tile is ready (and with it the P_x^T buffer of this parity is free: the issuer
         // waited for the transposed P V of two such tiles back)
         ok = __all_sync(0xffffffffu, mbar_wait(bar_sx_full + 8 * (gx & 1), (gx >> 1) & 1, abort_flag));
@@ -539,7 +573,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         // Exponents against the reference.  A tile that outgrows it (and the first tile, which has no
         // reference yet) takes the slow path; the four warps vote.
         float tx[kXMax];
-        bool over = (j == 0);
+        bool over = (jj == 0);
 #pragma unroll
         for (int i = 0; i < kXMax; ++i) {
           tx[i] = kv_live ? fmaf(__uint_as_float(sx[i]), c2, -mref[i]) : -INFINITY;
@@ -573,8 +607,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           for (int i = 0; i < kXMax; ++i) {
             const float c = fmaxf(fmaxf(xcol_s[0 * kXMax + i], xcol_s[1 * kXMax + i]),
                                   fmaxf(xcol_s[2 * kXMax + i], xcol_s[3 * kXMax + i]));
-            const float m_new = (j == 0) ? c : fmaxf(mref[i], c);
-            fx[i] = (j == 0) ? 0.f : ex2_approx(mref[i] - m_new);
+            const float m_new = (jj == 0) ? c : fmaxf(mref[i], c);
+            fx[i] = (jj == 0) ? 0.f : ex2_approx(mref[i] - m_new);
             lx[i] *= fx[i];
             mref[i] = m_new;
             tx[i] = kv_live ? fmaf(__uint_as_float(sx[i]), c2, -m_new) : -INFINITY;
@@ -582,7 +616,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           // xcol_s is reused by the next exchange: nobody may still be reading it
           ok = sync_y();
           if (!ok) break;
-          if (j > 0) {
+          if (jj > 0) {
             // O_x^T must be quiescent: the previous transposed P V has completed
             ok = __all_sync(0xffffffffu,
                             mbar_wait(bar_pvx_done + 8 * ((gx - 1) & 1), ((gx - 1) >> 1) & 1, abort_flag));
@@ -612,7 +646,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         if (lane == 0) mbar_arrive(bar_px_full + 8 * (gx & 1));
       }
       if (!ok) break;
-      gx0 += n_tiles;
+      gx0 += nt_cur;
       // ---- epilogue: column sums over all keys, then O_x^T / sum ----
 #pragma unroll
       for (int i = 0; i < kXMax; ++i) {
@@ -640,7 +674,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       // xcol_s is free again only when everyone has read it
       ok = sync_y();
       if (!ok) break;
-      __nv_bfloat16 *outp = reinterpret_cast<__nv_bfloat16 *>(prm.out) + it.b * prm.out_stride[0];
+      __nv_bfloat16 *outp = reinterpret_cast<__nv_bfloat16 *>(prm.out) + (kSplit ? it.split * prm.out_split_stride : 0) + it.b * prm.out_stride[0];
 #pragma unroll
       for (int i = 0; i < kXMax; ++i) {
         if (i < it.x_rows) {
@@ -649,7 +683,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           outp[hq * prm.out_stride[1] + (long long)ii * prm.out_stride[2] + row] =
               __float2bfloat16_rn(__uint_as_float(ox[i]) / lx[i]);
           if (prm.lse && row == 0)
-            prm.lse[((long long)it.b * prm.Hq + hq) * prm.Lq + ii] = (mref[i] + log2f(lx[i])) * kLn2;
+            prm.lse[(kSplit ? it.split * prm.lse_split_stride : 0) + ((long long)it.b * prm.Hq + hq) * prm.Lq + ii] = (mref[i] + log2f(lx[i])) * kLn2;
         }
       }
     }
@@ -666,13 +700,17 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     (void)tracer;
     bool ok = true;
     int g0 = 0, k = 0;
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
-      const Item it = decode_item(prm, item);
+    int nt_cur = 0;  // KV tiles of the current item that this CTA processes
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += nt_cur) {
+      const int j_lo = kSplit ? decode_item<kSplit>(prm, item).t0 : 0;
+      nt_cur = kSplit ? decode_item<kSplit>(prm, item).nt : n_tiles;
+      const Item it = decode_item<kSplit>(prm, item);
       const bool live = row < it.m_rows;
       float m_used = -INFINITY;  // maximum the probabilities are expressed against (log2 units)
       float l_sum = 0.f;         // this thread's half of the row sum
-      for (int j = 0; j < n_tiles; ++j) {
-        const int g = g0 + j;
+      for (int jj = 0; jj < nt_cur; ++jj) {
+        const int j = j_lo + jj;
+        const int g = g0 + jj;
         ok = mbar_wait(bar_s_full + 8 * (g & 1), (g >> 1) & 1, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -716,7 +754,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           factor = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_tile);
           m_used = m_tile;
         }
-        const bool warp_rescales = __any_sync(0xffffffffu, live && factor != 1.f) && (j > 0);
+        const bool warp_rescales = __any_sync(0xffffffffu, live && factor != 1.f) && (jj > 0);
         l_sum *= factor;
         float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
         const float neg_m = -m_used;
@@ -781,7 +819,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         const int R = it.mt * kBlockM + row;
         const int hq = it.hk * prm.G + R / prm.Lq, i = R % prm.Lq;
         const float inv = 1.f / l_sum;
-        __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(prm.out) + it.b * prm.out_stride[0] +
+        __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(prm.out) + (kSplit ? it.split * prm.out_split_stride : 0) + it.b * prm.out_stride[0] +
                               hq * prm.out_stride[1] + (long long)i * prm.out_stride[2] + kOCols * half;
 #pragma unroll
         for (int c = 0; c < kOCols; c += 8) {
@@ -792,7 +830,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
           *reinterpret_cast<uint4 *>(orow + c) = w;
         }
-        if (prm.lse && half == 0) prm.lse[((long long)it.b * prm.Hq + hq) * prm.Lq + i] = (m_used + log2f(l_sum)) * kLn2;
+        if (prm.lse && half == 0)
+          prm.lse[(kSplit ? it.split * prm.lse_split_stride : 0) + ((long long)it.b * prm.Hq + hq) * prm.Lq + i] = (m_used + log2f(l_sum)) * kLn2;
       }
     }
     timed_out = !ok;
@@ -810,6 +849,90 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
+// Stacked query rows of one KV head: full 128-row tiles, and a remainder that either rides along with the
+// last full tile (1..kXMax rows, D = 128) or gets a tile of its own.
+void tile_counts(const ds_attn_params &p, int &n_mtiles, int &x_rows) {
+  const long long rows_total = (long long)(p.Hq / p.Hkv) * p.Lq;
+  const int n_full = (int)(rows_total / kBlockM), rem = (int)(rows_total % kBlockM);
+  if (p.D == 128 && n_full >= 1 && rem >= 1 && rem <= kXMax) {
+    n_mtiles = n_full;
+    x_rows = rem;
+  } else {
+    n_mtiles = n_full + (rem ? 1 : 0);
+    x_rows = 0;
+  }
+}
+
+// Few work items (small batches) leave most SMs idle: split the KV tiles of every item over several CTAs.
+struct SplitPlan {
+  int splits, tiles_per_split;
+  size_t out_bytes, lse_bytes;  // partial results in the workspace
+};
+SplitPlan choose_splits(const ds_attn_params &p) {
+  int n_mtiles, x_rows;
+  tile_counts(p, n_mtiles, x_rows);
+  const int n_tiles = (p.P + kBlockN - 1) / kBlockN + (p.Lq + kBlockN - 1) / kBlockN;
+  const long long base = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv * n_mtiles;
+  int s = 1;
+  if (base > 0 && base * 2 <= sm_count() && n_tiles >= 4) {
+    s = (int)(sm_count() / base);
+    if (s > n_tiles / 2) s = n_tiles / 2;
+    if (s > 8) s = 8;
+  }
+  SplitPlan sp;
+  sp.tiles_per_split = (n_tiles + s - 1) / s;
+  // the merge is a second launch and every split fetches the queries again, measured to cost what about
+  // six KV tiles take: split only when it takes at least eight tiles off the critical path
+  if (n_tiles - sp.tiles_per_split < 8) sp.tiles_per_split = n_tiles;
+  sp.splits = (n_tiles + sp.tiles_per_split - 1) / sp.tiles_per_split;
+  const size_t rows = (size_t)p.B * p.Hq * p.Lq;
+  sp.out_bytes = sp.splits > 1 ? ((size_t)sp.splits * rows * p.D * 2 + 255) / 256 * 256 : 0;
+  sp.lse_bytes = sp.splits > 1 ? (size_t)sp.splits * rows * 4 : 0;
+  return sp;
+}
+
+// Merges the partial results of a split launch: out = sum_s w_s part_s / sum_s w_s with w_s = exp(lse_s - max lse).
+// One warp per (sequence, head, row).
+template <int D>
+__global__ void __launch_bounds__(256) attn_combine_kernel(const __nv_bfloat16 *__restrict__ part, const float *__restrict__ plse,
+                                                           int splits, long long out_split_stride, long long lse_split_stride,
+                                                           int B, int Hq, int Lq, __nv_bfloat16 *__restrict__ out,
+                                                           long long os0, long long os1, long long os2, float *__restrict__ lse,
+                                                           const int32_t *__restrict__ seq_list, int n_seq,
+                                                           const int32_t *__restrict__ n_seq_dev) {
+  int n_live = B;
+  if (seq_list != nullptr) {
+    n_live = n_seq;
+    if (n_seq_dev != nullptr) n_live = max(0, min(n_live, *n_seq_dev));
+  }
+  const long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= (long long)n_live * Hq * Lq) return;
+  const int lane = threadIdx.x & 31;
+  const int i = (int)(r % Lq), hq = (int)((r / Lq) % Hq);
+  int b = (int)(r / ((long long)Lq * Hq));
+  if (seq_list != nullptr) b = min(max(seq_list[b], 0), B - 1);
+  const long long prow = ((long long)b * Hq + hq) * Lq + i;
+  float m = -INFINITY;
+  for (int s = 0; s < splits; ++s) m = fmaxf(m, plse[s * lse_split_stride + prow]);
+  constexpr int kPer = D / 32;  // consecutive elements per lane
+  float acc[kPer];
+#pragma unroll
+  for (int c = 0; c < kPer; ++c) acc[c] = 0.f;
+  float wsum = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const float w = __expf(plse[s * lse_split_stride + prow] - m);
+    wsum += w;
+    const __nv_bfloat16 *src = part + s * out_split_stride + prow * D + lane * kPer;
+#pragma unroll
+    for (int c = 0; c < kPer; ++c) acc[c] += w * __bfloat162float(src[c]);
+  }
+  const float inv = 1.f / wsum;
+  __nv_bfloat16 *dst = out + b * os0 + hq * os1 + (long long)i * os2 + lane * kPer;
+#pragma unroll
+  for (int c = 0; c < kPer; ++c) dst[c] = __float2bfloat16_rn(acc[c] * inv);
+  if (lse != nullptr && lane == 0) lse[prow] = m + __logf(wsum);
+}
+
 template <int D>
 int prepare_d(const ds_attn_params &p, AttnPrepared &out) {
   static_assert(sizeof(TcParams) <= sizeof(out.kernel_params), "parameter struct does not fit the plan");
@@ -819,18 +942,26 @@ int prepare_d(const ds_attn_params &p, AttnPrepared &out) {
   out.p = p;
   out.grid = 0;
   if (!fill_common(prm, p)) return DS_ERR_CUDA;
-  // stacked query rows of one KV head: full 128-row tiles, and a remainder that either rides along
-  // with the last full tile (1..kXMax rows, D = 128) or gets a tile of its own
-  const long long rows_total = (long long)prm.G * p.Lq;
-  const int n_full = (int)(rows_total / kBlockM), rem = (int)(rows_total % kBlockM);
-  if (D == 128 && n_full >= 1 && rem >= 1 && rem <= kXMax) {
-    prm.n_mtiles = n_full;
-    prm.x_rows = rem;
-  } else {
-    prm.n_mtiles = n_full + (rem ? 1 : 0);
-    prm.x_rows = 0;
+  tile_counts(p, prm.n_mtiles, prm.x_rows);
+  const int n_tiles = (p.P + kBlockN - 1) / kBlockN + (p.Lq + kBlockN - 1) / kBlockN;
+  prm.splits = 1;
+  prm.tiles_per_split = n_tiles;
+  prm.n_tiles = n_tiles;
+  const SplitPlan sp = choose_splits(p);
+  if (sp.splits > 1 && p.workspace != nullptr && (reinterpret_cast<uintptr_t>(p.workspace) & 255) == 0 &&
+      p.workspace_bytes >= sp.out_bytes + sp.lse_bytes) {
+    // partial results, one dense [B][Hq][Lq][D] copy (and [B][Hq][Lq] log-sum-exp) per split, in the workspace
+    prm.splits = sp.splits;
+    prm.tiles_per_split = sp.tiles_per_split;
+    prm.out = p.workspace;
+    prm.out_stride[0] = (long long)p.Hq * p.Lq * p.D;
+    prm.out_stride[1] = (long long)p.Lq * p.D;
+    prm.out_stride[2] = p.D;
+    prm.out_split_stride = (long long)p.B * p.Hq * p.Lq * p.D;
+    prm.lse = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(p.workspace) + sp.out_bytes);
+    prm.lse_split_stride = (long long)p.B * p.Hq * p.Lq;
   }
-  const long long n_items = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv * prm.n_mtiles;  // upper bound with a device count
+  const long long n_items = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv * prm.n_mtiles * prm.splits;  // upper bound with a device count
   if (n_items > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   prm.n_items = (int)n_items;
   out.grid = (int)(n_items < sm_count() ? n_items : sm_count());
@@ -841,10 +972,26 @@ template <int D>
 int launch_prepared_d(const AttnPrepared &a, cudaStream_t stream) {
   if (a.grid == 0) return DS_OK;
   // the attribute is per device: set it at every launch (cheap)
-  DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes));
-  attn_tc_kernel<D><<<a.grid, kNumThreads, Geo<D>::kSmemBytes, stream>>>(*reinterpret_cast<const TcParams *>(a.kernel_params));
+  const TcParams &prm = *reinterpret_cast<const TcParams *>(a.kernel_params);
+  if (prm.splits > 1) {
+    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes));
+    attn_tc_kernel<D, true><<<a.grid, kNumThreads, Geo<D>::kSmemBytes, stream>>>(prm);
+  } else {
+    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes));
+    attn_tc_kernel<D, false><<<a.grid, kNumThreads, Geo<D>::kSmemBytes, stream>>>(prm);
+  }
   DS_CUDA_OK(cudaGetLastError());
   note_launch(1);
+  if (prm.splits > 1) {
+    const ds_attn_params &p = a.p;
+    const long long rows = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hq * p.Lq;
+    attn_combine_kernel<D><<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(
+        reinterpret_cast<const __nv_bfloat16 *>(prm.out), prm.lse, prm.splits, prm.out_split_stride, prm.lse_split_stride, p.B,
+        p.Hq, p.Lq, reinterpret_cast<__nv_bfloat16 *>(p.out), p.out_stride[0], p.out_stride[1], p.out_stride[2], p.lse,
+        p.seq_list, p.n_seq, p.seq_list ? p.n_seq_dev : nullptr);
+    DS_CUDA_OK(cudaGetLastError());
+    note_launch(1);
+  }
   return DS_OK;
 }
 
@@ -932,7 +1079,10 @@ bool attn_tc_supported(const ds_attn_params &p) {
   return true;
 }
 
-size_t attn_tc_workspace_bytes(const ds_attn_params &) { return 0; }
+size_t attn_tc_workspace_bytes(const ds_attn_params &p) {
+  const SplitPlan sp = choose_splits(p);
+  return sp.out_bytes + sp.lse_bytes;
+}
 
 int prepare_attn_tc(const ds_attn_params &p, AttnPrepared &out) {
   return p.D == 128 ? prepare_d<128>(p, out) : prepare_d<64>(p, out);
