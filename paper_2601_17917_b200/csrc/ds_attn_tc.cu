@@ -725,9 +725,10 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         // columns past the end of a partial tile do not exist
         const int valid = (j < n_pre) ? min(kBlockN, prm.P - j * kBlockN) : min(kBlockN, prm.Lq - (j - n_pre) * kBlockN);
         if (valid < kBlockN) {
+          // selects, not branches: the two half-warps see different limits
+          const int lim = valid - 64 * half;
 #pragma unroll
-          for (int c = 0; c < 64; ++c)
-            if (c + 64 * half >= valid) s[c] = 0xff800000u;  // -inf
+          for (int c = 0; c < 64; ++c) s[c] = (c >= lim) ? 0xff800000u : s[c];  // -inf: columns past the end of a partial tile
         }
         // row maximum: eight independent chains over this half, then the other half by shuffle
         float mx;

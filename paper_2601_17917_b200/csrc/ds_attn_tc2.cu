@@ -370,9 +370,10 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
           tmem_ld16x2_32<64>(s_base + 32, &s[32]);  // columns 64 half + 32..63
           tmem_wait_ld();
           if (valid < kBlockN) {
+            // selects, not branches: the two half-warps see different limits
+            const int lim = valid - 64 * half;
 #pragma unroll
-            for (int c = 0; c < 64; ++c)
-              if (c + 64 * half >= valid) s[c] = 0xff800000u;  // -inf: columns past the end of a partial tile
+            for (int c = 0; c < 64; ++c) s[c] = (c >= lim) ? 0xff800000u : s[c];  // -inf: columns past the end of a partial tile
           }
           float mx;
           {
