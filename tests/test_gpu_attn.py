@@ -335,12 +335,12 @@ def test_plan_launches_repeat_the_one_shot_call(path, dtype, monkeypatch):
     del plan
 
 
-@pytest.mark.parametrize("P,Lq", [(1500, 97), (2048, 129), (4096, 65), (1400, 136)])
-def test_few_work_items_split_over_the_keys(P, Lq, monkeypatch):
+@pytest.mark.parametrize("P,Lq,D", [(1500, 97, 128), (2048, 129, 128), (4096, 65, 128), (1400, 136, 128), (3000, 97, 64)])
+def test_few_work_items_split_over_the_keys(P, Lq, D, monkeypatch):
     # small batches: the KV tiles of an item are split over several CTAs and merged by a second kernel
     # (needs the workspace; without one the same call runs unsplit)
     monkeypatch.setenv("DS_ATTN_PATH", "tc")
-    B, Hq, Hkv, D, T = 2, 4, 2, 128, 1100
+    B, Hq, Hkv, T = 2, 4, 2, 1100
     g = torch.Generator().manual_seed(P + Lq)
     mk = lambda *sh: torch.randn(*sh, generator=g).to(torch.bfloat16).to(DEV)
     q, kt, vt = mk(B, Hq, T, D), mk(B, Hkv, T, D), mk(B, Hkv, T, D)
