@@ -89,9 +89,9 @@ namespace ds {
 namespace {
 // Several M-tiles per KV head (wide windows, the unpruned reference, a cache-refresh step): the two-tile
 // kernel fetches every KV tile once for a pair of M-tiles and keeps the softmax warps busy on one tile while
-// the tensor pipe works for the other.  Measured per work item it costs about 1.8 single tiles for a full pair
-// and 1.6 for a lone tile (no second S buffer to run ahead with), so it pays when the pairs are mostly full
-// and the number of rounds over the SMs does not grow.
+// the tensor pipe works for the other.  Measured per work item it costs about 1.85 single tiles for a full pair
+// and 1.05 for a pair with one tile (which alternates between the two S buffers like the one-tile kernel), so it
+// pays when the number of rounds over the SMs does not grow.
 bool two_tile_kernel_pays(const ds_attn_params &p) {
   const long long rows = (long long)(p.Hq / p.Hkv) * p.Lq;
   const long long n_full = rows / 128, rem = rows % 128;
@@ -102,7 +102,7 @@ bool two_tile_kernel_pays(const ds_attn_params &p) {
   const long long heads = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv, sms = sm_count();
   const double rounds1 = (double)((heads * n_mt1 + sms - 1) / sms);
   const double rounds2 = (double)((heads * n_pr + sms - 1) / sms);
-  const double pair_cost = (1.8 * (double)(n_mt / 2) + 1.6 * (double)(n_mt % 2)) / (double)n_pr;
+  const double pair_cost = (1.85 * (double)(n_mt / 2) + 1.05 * (double)(n_mt % 2)) / (double)n_pr;
   return rounds2 * pair_cost < 0.97 * rounds1;
 }
 

@@ -49,7 +49,7 @@ struct Geo2 {
   static constexpr int kOffRing = 2 * kTileBytes;
   static constexpr int kOffBar = kOffRing + kSlots * kTileBytes;
   // barriers: q_full, q_free, s_full[2], p_full[2], o_full, o_free[2], slot_full[kSlots], slot_empty[kSlots]
-  static constexpr int kNumBars = 9 + 2 * kSlots;
+  static constexpr int kNumBars = 11 + 2 * kSlots;   // + pv_done[2] (single-tile items)
   static constexpr int kOffIdx = kOffBar + 8 * kNumBars;
   static constexpr int kOffIdxQ = kOffIdx + 4 * 128;
   static constexpr int kOffIdxCache = kOffIdxQ + 4 * 128;
@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
   const uint32_t bar_o_free = bar0 + 56;  // [2] by M-tile
   const uint32_t bar_slot_full = bar0 + 72;
   const uint32_t bar_slot_empty = bar_slot_full + 8 * G_::kSlots;
+  const uint32_t bar_pv_done = bar_slot_empty + 8 * G_::kSlots;  // [2] by S buffer, items with one M-tile only
   int32_t *idx_s = reinterpret_cast<int32_t *>(smem + G_::kOffIdx);
   int32_t *idxq_s = reinterpret_cast<int32_t *>(smem + G_::kOffIdxQ);
   volatile uint32_t *tmem_base_s = reinterpret_cast<volatile uint32_t *>(smem + G_::kOffMisc);
@@ -115,6 +116,8 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
     mbar_init(bar_o_full, 1);
     mbar_init(bar_o_free, 8);
     mbar_init(bar_o_free + 8, 8);
+    mbar_init(bar_pv_done, 1);
+    mbar_init(bar_pv_done + 8, 1);
     for (int s = 0; s < G_::kSlots; ++s) {
       mbar_init(bar_slot_full + 8 * s, 1);
       mbar_init(bar_slot_empty + 8 * s, 1);
@@ -267,33 +270,34 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
     const uint64_t dv0 = smem_desc(sbase + G_::kOffRing, kChunkBytes, 1024);  // V tile, MN-major
     bool ok = true;
     int g0 = 0, k = 0;
-    int gb0 = 0;  // tiles of the items before this one in which M-tile b existed (phase count of its barriers)
-    // S_x = Q_x K(g)^T for M-tile x of the current item
-    auto issue_qk = [&](int x, int g, bool commit_k, bool last) {
+    int ua = 0, ub = 0;  // uses of the S_a / S_b buffers (phases of their barriers) before the current item
+    // S[sx] = Q_qx K(g)^T
+    auto issue_qk = [&](int sx, int qx, int g, bool commit_k, bool last) {
       const int fill = 2 * g, slot = fill % G_::kSlots;
       if (elect_one()) {
         const uint64_t dk = dk0 + (uint64_t)((slot * G_::kTileBytes) >> 4);
-        const uint64_t dq = dq0 + (uint64_t)((x * G_::kTileBytes) >> 4);
+        const uint64_t dq = dq0 + (uint64_t)((qx * G_::kTileBytes) >> 4);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = ((ks / 4) * kChunkBytes + (ks % 4) * 32) >> 4;
-          umma_ss(tm + G_::kTmemS + 128 * x, dq + off, dk + off, idesc_qk, ks > 0);
+          umma_ss(tm + G_::kTmemS + 128 * sx, dq + off, dk + off, idesc_qk, ks > 0);
         }
-        umma_commit(bar_s_full + 8 * x);
+        umma_commit(bar_s_full + 8 * sx);
         if (commit_k) umma_commit(bar_slot_empty + 8 * slot);
         if (last) umma_commit(bar_q_free);
       }
       __syncwarp();
     };
-    // O_x += P_x V(g)
-    auto issue_pv = [&](int x, int g, bool first, bool commit_v, bool last) {
+    // O[ox] += P[sx] V(g)
+    auto issue_pv = [&](int sx, int ox, int g, bool first, bool commit_v, bool last, bool commit_done) {
       const int fill = 2 * g + 1, slot = fill % G_::kSlots;
       if (elect_one()) {
         const uint64_t dv = dv0 + (uint64_t)((slot * G_::kTileBytes) >> 4);
 #pragma unroll
         for (int ks = 0; ks < kBlockN / 16; ++ks)
-          umma_ts(tm + G_::kTmemO + 128 * x, tm + G_::kTmemS + 128 * x + ks * 8, dv + ((ks * 2048) >> 4), idesc_pv,
+          umma_ts(tm + G_::kTmemO + 128 * ox, tm + G_::kTmemS + 128 * sx + ks * 8, dv + ((ks * 2048) >> 4), idesc_pv,
                   (!first || ks > 0) ? 1u : 0u);
+        if (commit_done) umma_commit(bar_pv_done + 8 * sx);
         if (commit_v) umma_commit(bar_slot_empty + 8 * slot);
         if (last) umma_commit(bar_o_full);
       }
@@ -302,6 +306,36 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += n_tiles) {
       const bool has_b = decode_item2(prm, item).rows_b > 0;
       ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full, k & 1, abort_flag));
+      if (!has_b) {
+        // One M-tile only: its KV tiles alternate between the two S buffers, so that Q K^T of tile j + 1 runs
+        // while tile j is in the softmax (the order of the one-tile kernel): Q K^T(0), Q K^T(1), P V(0),
+        // Q K^T(2), P V(1), ...  Every P V signals pv_done of its buffer (the lazy rescale of tile j + 1
+        // needs P V(j) complete, and here "S(j + 1) complete" does not say so).
+        for (int j = -1; j < n_tiles && ok; ++j) {
+          if (j + 1 < n_tiles) {
+            const int g = g0 + j + 1, fill = 2 * g, slot = fill % G_::kSlots, use = fill / G_::kSlots;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_slot_full + 8 * slot, use & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            issue_qk((j + 1) & 1, 0, g, true, j + 1 == n_tiles - 1);
+          }
+          if (j >= 0) {
+            const int g = g0 + j, fill = 2 * g + 1, slot = fill % G_::kSlots, use = fill / G_::kSlots;
+            const int sx = j & 1, px = (sx ? ub : ua) + (j >> 1);
+            bool w = mbar_wait2(bar_slot_full + 8 * slot, use & 1, bar_p_full + 8 * sx, px & 1, abort_flag);
+            if (j == 0 && k > 0) w = w && mbar_wait(bar_o_free, (k - 1) & 1, abort_flag);
+            if (!__all_sync(0xffffffffu, w)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            issue_pv(sx, 0, g, j == 0, true, j == n_tiles - 1, true);
+          }
+        }
+        ua += (n_tiles + 1) / 2;
+        ub += n_tiles / 2;
+        continue;
+      }
       for (int j = 0; j <= n_tiles && ok; ++j) {
         const int g = g0 + j;  // tile whose Q K^T is issued; P V is issued for tile g - 1
         if (j < n_tiles) {
@@ -310,12 +344,11 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
           if (!ok) break;
         }
         for (int x = 0; x < 2 && ok; ++x) {
-          if (x == 1 && !has_b) break;
           if (j > 0) {
             // P_x of the previous tile is in TMEM and its V tile has landed; the epilogue of the previous item
             // has read O_x before the first P V of this one overwrites it
             const int gp = g - 1, fill = 2 * gp + 1, slot = fill % G_::kSlots, use = fill / G_::kSlots;
-            const int px = (x ? gb0 : g0) + j - 1;  // tiles M-tile x has seen before this P
+            const int px = (x ? ub : ua) + j - 1;  // uses of S_x before this P
             bool w = mbar_wait2(bar_slot_full + 8 * slot, use & 1, bar_p_full + 8 * x, px & 1, abort_flag);
             if (j == 1 && k > 0) w = w && mbar_wait(bar_o_free + 8 * x, (k - 1) & 1, abort_flag);
             if (!__all_sync(0xffffffffu, w)) {
@@ -323,17 +356,16 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
               break;
             }
             tc_fence_after();
-            const bool last_x = (x == 1) || !has_b;
-            issue_pv(x, gp, j == 1, last_x, last_x && j == n_tiles);
+            issue_pv(x, x, gp, j == 1, x == 1, x == 1 && j == n_tiles, false);
           }
           if (j < n_tiles) {
             tc_fence_after();
-            const bool last_x = (x == 1) || !has_b;
-            issue_qk(x, g, last_x, last_x && j == n_tiles - 1);
+            issue_qk(x, x, g, x == 1, x == 1 && j == n_tiles - 1);
           }
         }
       }
-      if (has_b) gb0 += n_tiles;
+      ua += n_tiles;
+      ub += n_tiles;
     }
     timed_out = !ok;
   } else {
@@ -348,10 +380,12 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
     const float c2 = prm.scale_log2;
     constexpr int kOCols = D / 2;                          // accumulator columns per thread
     bool ok = true;
-    int ga0 = 0, gb0 = 0, k = 0;  // tiles M-tile a / b have seen before the current item (phase counts of their barriers)
+    int ga0 = 0, gb0 = 0, k = 0;  // uses of the S_a / S_b buffers before the current item (phase counts of their barriers)
+    int da0 = 0, db0 = 0;         // the same, counting single-tile items only (phases of pv_done)
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k) {
       const Item2 it = decode_item2(prm, item);
       const int n_x = it.rows_b > 0 ? 2 : 1;
+      const bool lone = n_x == 1;  // one M-tile: its KV tiles alternate between the two S buffers
       float m_used[2] = {-INFINITY, -INFINITY};  // maximum the probabilities are expressed against (log2 units)
       float l_sum[2] = {0.f, 0.f};               // this thread's half of the row sum
       for (int j = 0; j < n_tiles && ok; ++j) {
@@ -360,11 +394,12 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
         for (int x = 0; x < 2; ++x) {
           if (x >= n_x) break;
           const bool live = row < (x ? it.rows_b : it.rows_a);
-          const int gx = (x ? gb0 : ga0) + j;
-          ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * x, gx & 1, abort_flag));
+          const int sx = lone ? (j & 1) : x;  // S buffer of this tile
+          const int gx = (sx ? gb0 : ga0) + (lone ? (j >> 1) : j);
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * sx, gx & 1, abort_flag));
           if (!ok) break;
           tc_fence_after();
-          const uint32_t s_base = lane_base + G_::kTmemS + 128 * x, o_base = lane_base + G_::kTmemO + 128 * x;
+          const uint32_t s_base = lane_base + G_::kTmemS + 128 * sx, o_base = lane_base + G_::kTmemO + 128 * x;
           uint32_t s[64];
           tmem_ld16x2_32<64>(s_base, &s[0]);        // columns 64 half + 0..31
           tmem_ld16x2_32<64>(s_base + 32, &s[32]);  // columns 64 half + 32..63
@@ -400,8 +435,15 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
           const bool warp_rescales = __any_sync(0xffffffffu, live && factor != 1.f) && (j > 0);
           l_sum[x] *= factor;
           if (warp_rescales) {
-            // S of this tile being complete means every MMA issued before its Q K^T has completed, the
-            // previous P V of this M-tile among them: O_x is quiescent
+            // With two M-tiles, S of this tile being complete means every MMA issued before its Q K^T has
+            // completed, the previous P V of this M-tile among them: O_x is quiescent.  With one M-tile the
+            // previous P V was issued after this Q K^T and has a barrier of its own.
+            if (lone) {
+              const int sp = (j - 1) & 1, gp = (sp ? db0 : da0) + ((j - 1) >> 1);
+              ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + 8 * sp, gp & 1, abort_flag));
+              if (!ok) break;
+              tc_fence_after();
+            }
 #pragma unroll
             for (int cb = 0; cb < kOCols; cb += 32) {
               uint32_t o[32];
@@ -435,7 +477,7 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
           tmem_wait_st();
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_p_full + 8 * x);
+          if (lane == 0) mbar_arrive(bar_p_full + 8 * sx);
         }
       }
       if (!ok) break;
@@ -475,8 +517,12 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
           if (prm.lse && half == 0) prm.lse[((long long)it.b * prm.Hq + hq) * prm.Lq + i] = (m_used[x] + log2f(l_row)) * kLn2;
         }
       }
-      ga0 += n_tiles;
-      if (n_x == 2) gb0 += n_tiles;
+      ga0 += lone ? (n_tiles + 1) / 2 : n_tiles;
+      gb0 += lone ? n_tiles / 2 : n_tiles;
+      if (lone) {
+        da0 += (n_tiles + 1) / 2;
+        db0 += n_tiles / 2;
+      }
     }
     timed_out = !ok;
   }
@@ -504,7 +550,22 @@ int prepare2_d(const ds_attn_params &p, AttnPrepared &out) {
   const long long n_items = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv * prm.n_pairs;  // upper bound with a device count
   if (n_items > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   prm.n_items = (int)n_items;
-  out.grid = (int)(n_items < sm_count() ? n_items : sm_count());
+  int grid = (int)(n_items < sm_count() ? n_items : sm_count());
+  // An odd number of M-tiles leaves a pair with one tile, about half the work of a full pair.  CTA c takes the
+  // items c, c + grid, ...; the pair number is the fastest index of an item, so a grid that shares a factor with
+  // the number of pairs would hand some CTAs nothing but full pairs: keep the two coprime.
+  if ((rows_total + kBlockM - 1) / kBlockM % 2 == 1 && prm.n_pairs > 1 && n_items > grid) {
+    auto gcd = [](int a, int b) {
+      while (b) {
+        const int t = a % b;
+        a = b;
+        b = t;
+      }
+      return a;
+    };
+    while (grid > 1 && gcd(grid, prm.n_pairs) != 1) --grid;
+  }
+  out.grid = grid;
   return DS_OK;
 }
 
