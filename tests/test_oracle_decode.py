@@ -114,3 +114,21 @@ def test_invariants_of_the_procedure(alpha):
             m = e["masked"][b] == 1
             above = m & (c >= tau)
             assert np.array_equal(newly[b], above) if above.any() else newly[b].sum() == 1
+
+
+def test_ratio_over_the_query_counts_the_retained_suffix_rows():
+    # Eq. 10 with r_mask taken over the whole query: K = 2 block positions plus e = 2 retained suffix rows that are
+    # always masked.  Two masked: r = 4/4, tau = tau0; one masked: r = 3/4, tau = tau0 (1 - alpha / 4).
+    ln = np.log
+    z = {
+        (0, 0): np.array([[[ln(18.0), 0, 0], [0, ln(2.0), 0]]]),   # confidences 0.9 and 0.5 against tau = 0.85
+        (0, 1): np.array([[[0, 0, 5.0], [0, 0, ln(8.0)]]]),        # 0.8 against tau = 0.85 * 0.9 = 0.765: accepted
+    }
+    tr = []
+    r = oracle.decode(_table_fn(z), 1, 2, 2, tau0=0.85, alpha=0.4, mask_id=MASK, extra_fn=lambda n: 2, trace=tr)
+    assert [round(float(e["tau"][0]), 6) for e in tr] == [0.85, 0.765]
+    assert r["x"].tolist() == [[0, 2]] and r["steps"].tolist() == [2]
+    # with the block-only ratio the second threshold is 0.85 (1 - 0.4 / 2) = 0.68
+    tr2 = []
+    oracle.decode(_table_fn(z), 1, 2, 2, tau0=0.85, alpha=0.4, mask_id=MASK, trace=tr2)
+    assert [round(float(e["tau"][0]), 6) for e in tr2] == [0.85, 0.68]
