@@ -42,8 +42,10 @@ def sweep_window(device, base="long32-w64", windows=(0, 32, 64, 128, 256, 512, 1
     x = wl.attention_inputs(cfg0, device=device)
     scale = 1.0 / math.sqrt(cfg0.D)
     esz = 2 if cfg0.dtype == "bf16" else 4
-    for keep_last in (True, False):
-        for w in windows:
+    # both variants of a window back to back, the long-running whole-suffix point last: a point measured right
+    # after seconds of dense work would see the power-capped clock, not its own
+    for w in windows:
+        for keep_last in (True, False):
             if w < 0 and not keep_last:
                 continue
             idx = retained_indices(cfg0.gen, cfg0.K, 0, w, keep_last)
