@@ -123,6 +123,37 @@ def test_confidence_and_select_argument_validation(L):
     assert L.ds_unmask_select(None, None) == ds.DS_ERR_INVALID_ARG
 
 
+def test_loop_control_entry_points_validate_without_a_gpu(L):
+    fake = ctypes.c_void_p(0x7f0000000000)
+    # plans: an invalid description gives the error of ds_attn_pruned and no plan; destroying NULL is allowed
+    h = ctypes.c_void_p(0x1234)
+    assert L.ds_attn_plan_create(ctypes.byref(_attn(Lq=0)), ctypes.byref(h)) == ds.DS_ERR_INVALID_ARG
+    assert not h.value
+    assert L.ds_attn_plan_create(ctypes.byref(_attn()), None) == ds.DS_ERR_INVALID_ARG
+    assert L.ds_attn_plan_launch(None, None) == ds.DS_ERR_INVALID_ARG
+    L.ds_attn_plan_destroy(None)
+    # sequence lists
+    p = _attn()
+    p.seq_list, p.n_seq = 0x7f0000000000, p.B + 1
+    assert L.ds_attn_pruned(ctypes.byref(p), None) == ds.DS_ERR_INVALID_ARG
+    p.n_seq = -1
+    assert L.ds_attn_pruned(ctypes.byref(p), None) == ds.DS_ERR_INVALID_ARG
+    # rows listed on the device
+    assert L.ds_confidence_listed(fake, 1, 4, 100, 100, None, 4, fake, fake, fake, None, 0, None) == ds.DS_ERR_INVALID_ARG
+    assert L.ds_confidence_listed(fake, 1, 4, 100, 100, fake, 4, None, fake, fake, None, 0, None) == ds.DS_ERR_INVALID_ARG
+    assert L.ds_confidence_listed(fake, 1, 4, 100, 100, fake, 5, fake, fake, fake, None, 0, None) == ds.DS_ERR_INVALID_ARG
+    assert L.ds_confidence_listed(fake, 1, 4, 100, 100, fake, 0, fake, fake, fake, None, 0, None) == ds.DS_OK
+    # start of a block
+    b = ds._BlockParams()
+    assert L.ds_block_begin(None, None) == ds.DS_ERR_INVALID_ARG
+    assert L.ds_block_begin(ctypes.byref(b), None) == ds.DS_ERR_INVALID_ARG       # K = 0
+    b.B, b.K, b.active_cnt = 2, 32, 0x7f0000000000
+    assert L.ds_block_begin(ctypes.byref(b), None) == ds.DS_ERR_INVALID_ARG       # null arrays
+    b.masked_rows = 0x7f0000000000                                                  # rows without their count
+    assert L.ds_block_begin(ctypes.byref(b), None) == ds.DS_ERR_INVALID_ARG
+    assert L.ds_last_cuda_error() == 0 and L.ds_last_cuda_error_name() == b"cudaSuccess"
+
+
 def test_host_index_list_matches_oracle():
     for gen, K, c, w, last in [(256, 32, 0, 16, True), (256, 32, 0, 32, True), (1024, 32, 0, 64, True),
                                (4096, 64, 0, 0, False), (4096, 64, 0, 64, True), (4096, 64, 0, 256, True),
