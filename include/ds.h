@@ -56,10 +56,15 @@ typedef enum {
 } ds_status;
 
 /* bits OR-ed into the optional device status word */
-#define DS_DEV_INDEX 1u   /* an entry of idx was outside [0, T); it was clamped */
+#define DS_DEV_INDEX 1u   /* an entry of idx (or of a sequence list) was out of range and was clamped, or idx was not
+                             strictly ascending (its rows are then fetched one by one, in the order given) */
 #define DS_DEV_TIMEOUT 2u /* a bounded mbarrier wait expired; outputs of that CTA are invalid */
 
 typedef enum { DS_F32 = 0, DS_BF16 = 1 } ds_dtype;
+
+/* bf16 attention kernels: one 128-row query tile per work item (KV-stream bound shapes), or a pair of query
+ * tiles sharing every KV tile (several tiles per KV head: wide windows, GQA groups, a cache-refresh step). */
+typedef enum { DS_ATTN_KERNEL_AUTO = 0, DS_ATTN_KERNEL_ONE_TILE = 1, DS_ATTN_KERNEL_TWO_TILE = 2 } ds_attn_kernel;
 
 /* ------------------------------------------------------------------------
  * ds_attn_pruned  (Eq. 7, Eq. 8; "Dynamic Confidence Aware Parallel Decoding")
@@ -68,6 +73,9 @@ typedef enum { DS_F32 = 0, DS_BF16 = 1 } ds_dtype;
  * (Method, region split).  The "tail" is block + suffix, T rows.  The retained
  * set of Eq. 7 arrives as `idx`: Lq tail-relative row numbers, strictly
  * ascending (block rows first, then the window, then the trailing position).
+ * The kernels rely on the order to fetch runs of consecutive rows as one
+ * box: they check it, and a list that is not strictly ascending raises
+ * DS_DEV_INDEX and is served row by row exactly as written.
  * For every batch b and query head h, with KV head g = h / (Hq / Hkv):
  *
  *     Q~ = q_tail[b, h, idx[:], :]                          (Lq x D)
@@ -86,8 +94,11 @@ typedef enum { DS_F32 = 0, DS_BF16 = 1 } ds_dtype;
  * prefix pointers are then ignored).  idx is either one list shared by all
  * batches (idx_batch_stride = 0) or one per batch.
  *
- * Envelope: D in {64, 128} for the tensor-core bf16 path; the fp32 path takes
- * any D that is a multiple of 32 up to 256.  Hq % Hkv == 0.  1 <= Lq <= T.
+ * Envelope: DS_BF16 runs on the tensor cores and takes D in {64, 128} and
+ * scale > 0; DS_F32 runs on the CUDA cores and takes D in {32, 64, 128, 256}
+ * and any finite scale.  Hq % Hkv == 0.  1 <= Lq <= T.  B, Hq <= 65535.
+ * Anything else that is well formed returns DS_ERR_UNSUPPORTED: no request is
+ * rerouted to another kernel behind the caller's back.
  *
  * Workspace: ds_attn_pruned_workspace(p) bytes, 256-byte aligned; contents need
  * not be preserved between calls.  It is used when the call has few work
@@ -95,8 +106,10 @@ typedef enum { DS_F32 = 0, DS_BF16 = 1 } ds_dtype;
  * split over several CTAs, which leave normalised partial results and their
  * log-sum-exp in the workspace, and a second kernel merges them.  A call
  * without a (large enough) workspace is not an error; it runs unsplit.
- * Errors: DS_ERR_INVALID_ARG / DS_ERR_UNSUPPORTED / DS_ERR_WORKSPACE before
- * anything is launched; DS_ERR_CUDA if a launch fails.
+ * Errors: DS_ERR_INVALID_ARG / DS_ERR_UNSUPPORTED before anything is
+ * launched; DS_ERR_CUDA if a tensor-map encoding or a launch fails
+ * (ds_last_cuda_error tells which runtime error; for a refused encoding it
+ * reports cudaErrorInvalidValue).
  * ------------------------------------------------------------------------ */
 typedef struct {
   int32_t B, Hq, Hkv, D;
@@ -128,6 +141,10 @@ typedef struct {
   const int32_t *seq_list;
   int32_t n_seq;
   const int32_t *n_seq_dev;
+  /* Which bf16 kernel serves the call (ds_attn_kernel).  DS_ATTN_KERNEL_AUTO lets the library choose by
+   * shape; the other two values pin the choice (a caller that has timed both on its shapes, a test that
+   * wants each kernel on the same inputs).  Ignored for DS_F32.  Any other value: DS_ERR_INVALID_ARG. */
+  int32_t kernel;
 } ds_attn_params;
 
 /* HOST, pure: bytes of workspace ds_attn_pruned needs for *p (0 when none). */
@@ -181,8 +198,9 @@ DS_API int ds_confidence_listed(const void *logits, int32_t dtype, int64_t rows,
 /* ------------------------------------------------------------------------
  * ds_rope_gather  (Eq. 7 position ids, Eq. 8 pruned input, prefix-cache append)
  *
- * The suffix pruning keeps "the logical ordering of tokens via RoPE position
- * IDs": a retained row keeps the position it has in the full sequence.  This
+ * Pruned tokens keep their place in the sequence through their rotary
+ * position ids (Eq. 7 and the text around it): a retained row is rotated with
+ * the position it has in the full sequence, not with its rank in the list.  This
  * entry point takes the un-rotated projections of the whole tail and produces
  * what ds_attn_pruned consumes, compact and rotated.  For every batch b and
  * retained row i (tail row r = idx[i], absolute position pos = pos_offset + r):
@@ -227,10 +245,10 @@ DS_API int ds_rope_gather(const ds_rope_params *p, void *stream);
 /* ------------------------------------------------------------------------
  * ds_lmhead_confidence  (output projection + Eq. 4, fused)
  *
- * In the prediction forward the attention outputs are "processed by the
- * remaining model components to produce the prediction logits" (Method,
- * "Dynamic Confidence Aware Parallel Decoding"); the last of them is the output
- * projection z_r = W h_r.  This entry point computes, for every row r,
+ * After the attention, the rest of the model turns the hidden states into the
+ * prediction logits (Method, "Dynamic Confidence Aware Parallel Decoding"); the
+ * last of those components is the output projection z_r = W h_r.  This entry
+ * point computes, for every row r,
  *     z_rj    = sum_k hidden[r][k] * weight[j][k]          (j < V, fp32 accumulation)
  *     tok[r]  = lowest j with z_rj == max_j z_rj
  *     conf[r] = 1 / sum_j exp(z_rj - max_j z_rj)            (Eq. 4)
@@ -274,7 +292,9 @@ DS_API int ds_lmhead_confidence(const void *hidden, const void *weight, int64_t 
  * First call on a device: it looks up the device address of the scratch array
  * (a CUDA runtime query, remembered per device; the device that is current at
  * the call is the one set up).  Make that first call outside any stream
- * capture.
+ * capture.  The remembered address belongs to the device's current context:
+ * after cudaDeviceReset it is stale, and the process must not call this entry
+ * point on that device again.
  *
  * Sharing: every call on a device uses the same array, and the array keeps
  * the previous call's contents; the function clears the tickets it is about
@@ -346,9 +366,10 @@ DS_API int ds_unmask_select(const ds_select_params *p, void *stream);
 /* ------------------------------------------------------------------------
  * ds_block_begin  (Eq. 1, Eq. 2, block termination rule, early exit)
  *
- * Decoding proceeds block by block: when block n has no masked position left
- * "the model proceeds to decode block n+1", and once a sequence has predicted
- * EOS with high confidence "all subsequent blocks are skipped".  This entry
+ * Decoding proceeds block by block: a block whose positions are all unmasked
+ * is followed by the next one (end of Preliminary), and a sequence that has
+ * predicted EOS with high confidence decodes no further block ("Early Exit For
+ * Block Diffusion").  This entry
  * point prepares the device state of the next block from the per-sequence
  * early-exit flags, without the host looking at them:
  *     for b with eos_exit[b] == 0:  masked[b][:] = 1, x_block[b][:] = mask_id   (Eq. 1: K fresh [MASK])
@@ -378,6 +399,18 @@ DS_API int ds_block_begin(const ds_block_params *p, void *stream);
 /* ------------------------------------------------------------------------
  * Utilities
  * ------------------------------------------------------------------------ */
+/* Self-test of the bounded wait (no counterpart in the paper; the tensor-core kernels' failure handling).
+ * Every on-chip wait of the attention and projection kernels is a poll loop with a limit, after which the
+ * kernel raises DS_DEV_TIMEOUT and leaves in order.  This call runs that same wait, in a one-warp kernel, on
+ * a barrier nobody arrives on, with `poll_limit` polls (1 .. 65536; a few microseconds to milliseconds), so
+ * that a deployment can check the expiry path on its GPU without a real kernel having to fail:
+ *     *status   |= DS_DEV_TIMEOUT                      (optional device word)
+ *     report[0]  = 1  the wait gave up                  (optional device int32[3])
+ *     report[1]  = 1  the CTA-wide give-up flag was set
+ *     report[2]  = 1  after one arrival, a second wait on the same barrier succeeded
+ * The kernel always terminates and the context stays usable.  Errors: DS_ERR_INVALID_ARG (limit out of
+ * range, misaligned pointer), DS_ERR_CUDA. */
+DS_API int ds_selftest_bounded_wait(uint32_t poll_limit, uint32_t *status, int32_t *report, void *stream);
 /* Copies the device status word to *host_out (HOST) after synchronising `stream`. */
 DS_API int ds_read_status(const uint32_t *device_status, void *stream, uint32_t *host_out);
 /* HOST: static string for a ds_status value. */

@@ -15,11 +15,13 @@ Contents
   pin ``attn``: retaining every suffix position must reproduce it.
 * ``confidence`` (C, ``oracle_confidence``): Eq. 4.
 * ``rope_gather`` (C, ``oracle_rope_gather``): rotary encoding of the retained
-  rows with their original position ids (Eq. 7's "positional information ...
-  via RoPE position IDs") and their gather into compact Q/K/V.
+  rows with their original position ids (Eq. 7 and the text around it: pruned
+  tokens keep their place through their rotary position ids) and their gather
+  into compact Q/K/V.
 * ``lmhead_confidence`` (C, ``oracle_lmhead_confidence``): the output projection
-  (last of the "remaining model components" that turn attention outputs into
-  logits) composed with Eq. 4, logits kept in float64.
+  (the last of the components that turn attention outputs into logits,
+  Method, "Dynamic Confidence Aware Parallel Decoding") composed with Eq. 4,
+  logits kept in float64.
 * ``threshold`` / ``select`` (C, float32, contraction off): Eq. 10, Eq. 9, Eq. 5,
   block termination and the early-exit flag.
 * ``decode`` (Python loop over the above): the block-wise decoding procedure of
@@ -302,8 +304,8 @@ def decode(logits_fn, B: int, L: int, K: int, tau0: float, alpha: float, mask_id
     Eq. 4 gives confidences and tokens, Eq. 9-10 choose the positions to finalise, Eq. 5 updates them.
     Sequences whose block is finished are no longer processed (their logits are not looked at).
     Early exit: a sequence that finalised ``eos_id`` with confidence >= ``eos_tau`` finishes its current
-    block and skips every later block; the skipped blocks are filled with ``eos_id`` (the paper only says
-    the sequence "remains complete").
+    block and skips every later block; the skipped blocks are filled with ``eos_id`` (what they hold is not
+    stated in the paper).
     ``extra_fn(n)`` = number of retained suffix rows counted as masked in Eq. 10's ratio (None: 0).
 
     Returns dict(x [B, L] int32, steps [N] iterations spent on each block, seq_steps [B, N] iterations

@@ -233,10 +233,9 @@ int oracle_select(int B, int K, const float *conf, const int32_t *tok,
 /*
  * Output projection followed by Eq. 4, without storing the logits.
  *
- * In the prediction forward the attention output is "processed by the
- * remaining model components to produce the prediction logits" (Method,
- * "Dynamic Confidence Aware Parallel Decoding"); the last of those components
- * is the output projection z_r = W h_r.  Eq. 4 then reads c_r = max_j
+ * After the attention, the rest of the model turns the hidden states into the
+ * prediction logits (Method, "Dynamic Confidence Aware Parallel Decoding");
+ * the last of those components is the output projection z_r = W h_r.  Eq. 4 then reads c_r = max_j
  * softmax(z_r)_j and x^_r = argmax_j z_rj.  This function is that composition
  * written out: a plain matrix-vector product in double per row, then the same
  * max / lowest-index argmax / sum of exponentials as oracle_confidence.
@@ -285,8 +284,9 @@ int oracle_lmhead_confidence(const float *hidden, const float *weight, long rows
 /*
  * Rotary position encoding of the retained rows with their ORIGINAL position
  * ids, and their gather into compact buffers (Method, "Attenuation Guided
- * Suffix Modeling": the pruned suffix keeps "the logical ordering of tokens
- * via RoPE position IDs"; Eq. 7 names the retained set, Eq. 8 the pruned input).
+ * Suffix Modeling": pruned tokens keep their place in the sequence through
+ * their rotary position ids; Eq. 7 names the retained set, Eq. 8 the pruned
+ * input).
  *
  * For every batch b, head h and retained row i (tail row r = idx[i], absolute
  * position p = pos_offset + r), with half = D / 2 and, for d < half,

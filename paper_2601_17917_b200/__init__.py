@@ -20,14 +20,16 @@ __all__ = [
     "lib", "retained_indices", "ds_attn_pruned", "ds_attn_pruned_workspace", "ds_confidence",
     "ds_confidence_workspace", "ds_confidence_static", "ds_lmhead_confidence", "ds_lmhead_confidence_workspace",
     "ds_rope_gather", "ds_unmask_select", "ds_read_status", "ds_strerror", "ds_version",
-    "ds_launch_count", "ds_block_begin", "ds_confidence_listed", "AttnPlan",
+    "ds_launch_count", "ds_block_begin", "ds_confidence_listed", "AttnPlan", "ds_selftest_bounded_wait",
     "DsError", "DS_F32", "DS_BF16", "DS_DEV_INDEX", "DS_DEV_TIMEOUT",
+    "DS_ATTN_KERNEL_AUTO", "DS_ATTN_KERNEL_ONE_TILE", "DS_ATTN_KERNEL_TWO_TILE",
 ]
 
 DS_F32, DS_BF16 = 0, 1
 DS_OK, DS_ERR_INVALID_ARG, DS_ERR_UNSUPPORTED, DS_ERR_WORKSPACE, DS_ERR_CUDA, DS_ERR_STATIC_LIMIT = range(6)
 DS_CONFIDENCE_STATIC_MAX_ROWS = 4096
 DS_DEV_INDEX, DS_DEV_TIMEOUT = 1, 2
+DS_ATTN_KERNEL_AUTO, DS_ATTN_KERNEL_ONE_TILE, DS_ATTN_KERNEL_TWO_TILE = 0, 1, 2
 
 _LIB_PATH = Path(__file__).resolve().parent / "libds_b200.so"
 _lib = None
@@ -54,6 +56,7 @@ class _AttnParams(ctypes.Structure):
         ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t), ("status", ctypes.c_void_p),
         ("seq_list", ctypes.c_void_p), ("n_seq", ctypes.c_int32), ("n_seq_dev", ctypes.c_void_p),
+        ("kernel", ctypes.c_int32),
     ]
 
 
@@ -139,6 +142,8 @@ def lib() -> ctypes.CDLL:
         L.ds_unmask_select.argtypes = [ctypes.POINTER(_SelectParams), ctypes.c_void_p]
         L.ds_read_status.restype = ctypes.c_int
         L.ds_read_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
+        L.ds_selftest_bounded_wait.restype = ctypes.c_int
+        L.ds_selftest_bounded_wait.argtypes = [ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.ds_last_cuda_error.restype = ctypes.c_int
         L.ds_last_cuda_error_name.restype = ctypes.c_char_p
         L.ds_strerror.restype = ctypes.c_char_p
@@ -203,7 +208,7 @@ def retained_indices(gen_len: int, K: int, c: int, w_tokens: int, keep_last: boo
 
 
 def _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status,
-                 seq_list=None, n_seq=None, n_seq_dev=None):
+                 seq_list=None, n_seq=None, n_seq_dev=None, kernel=DS_ATTN_KERNEL_AUTO):
     B, Hq, T, D = q_tail.shape
     Hkv = k_tail.shape[1]
     P = 0 if k_prefix is None else k_prefix.shape[2]
@@ -242,27 +247,30 @@ def _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, ls
         p.seq_list = seq_list.data_ptr()
         p.n_seq = seq_list.numel() if n_seq is None else min(int(n_seq), seq_list.numel())
         p.n_seq_dev = n_seq_dev.data_ptr() if n_seq_dev is not None else None
+    p.kernel = int(kernel)
     return p
 
 
-def ds_attn_pruned_workspace(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out) -> int:
-    p = _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, None, None, None)
+def ds_attn_pruned_workspace(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out,
+                             kernel=DS_ATTN_KERNEL_AUTO) -> int:
+    p = _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, None, None, None, kernel=kernel)
     return int(lib().ds_attn_pruned_workspace(ctypes.byref(p)))
 
 
 def ds_attn_pruned(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out=None, lse=None,
-                   workspace=None, status=None, stream=None, seq_list=None, n_seq=None, n_seq_dev=None):
+                   workspace=None, status=None, stream=None, seq_list=None, n_seq=None, n_seq_dev=None,
+                   kernel=DS_ATTN_KERNEL_AUTO):
     """Pruned attention (Eq. 7-8).  q_tail [B,Hq,T,D]; k_tail, v_tail [B,Hkv,T,D];
     k_prefix, v_prefix [B,Hkv,P,D] or None; idx int32 [Lq] or [B,Lq] on the device.
     seq_list (int32, ascending batch numbers; its first n_seq entries, or as many as the device scalar
-    n_seq_dev says) restricts the call to those sequences.
+    n_seq_dev says) restricts the call to those sequences.  ``kernel`` pins the bf16 kernel (DS_ATTN_KERNEL_*).
     Returns ``out`` [B,Hq,Lq,D].  Allocates ``out``/``workspace`` with torch when not given."""
     _check_dev(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, out, lse, workspace, status, seq_list, n_seq_dev)
     B, Hq, T, D = q_tail.shape
     if out is None:
         out = torch.empty((B, Hq, idx.shape[-1], D), dtype=q_tail.dtype, device=q_tail.device)
     p = _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status,
-                     seq_list, n_seq, n_seq_dev)
+                     seq_list, n_seq, n_seq_dev, kernel)
     if workspace is None:
         need = int(lib().ds_attn_pruned_workspace(ctypes.byref(p)))
         if need:
@@ -280,13 +288,13 @@ class AttnPlan:
     (their contents are read at every launch).  ``out`` is allocated when not given."""
 
     def __init__(self, q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out=None, lse=None, workspace=None,
-                 status=None, seq_list=None, n_seq=None, n_seq_dev=None):
+                 status=None, seq_list=None, n_seq=None, n_seq_dev=None, kernel=DS_ATTN_KERNEL_AUTO):
         _check_dev(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, out, lse, workspace, status, seq_list, n_seq_dev)
         B, Hq, T, D = q_tail.shape
         if out is None:
             out = torch.empty((B, Hq, idx.shape[-1], D), dtype=q_tail.dtype, device=q_tail.device)
         p = _attn_params(q_tail, k_tail, v_tail, k_prefix, v_prefix, idx, scale, out, lse, workspace, status,
-                         seq_list, n_seq, n_seq_dev)
+                         seq_list, n_seq, n_seq_dev, kernel)
         if workspace is None:
             need = int(lib().ds_attn_pruned_workspace(ctypes.byref(p)))
             if need:
@@ -333,6 +341,8 @@ def ds_confidence(logits, row_list=None, conf=None, tok=None, workspace=None, st
         workspace = torch.empty(max(need, 1), dtype=torch.uint8, device=logits.device)
     if row_list is not None and row_list.dtype != torch.int32:
         raise TypeError("row_list must be int32")
+    if row_list is not None and row_list.numel() == 0:
+        return conf, tok      # no row listed: nothing is touched (a null list pointer would mean "all rows")
     rc = lib().ds_confidence(_ptr(logits), _dtype_code(logits), rows, V, logits.stride(0), _ptr(row_list),
                              0 if row_list is None else row_list.numel(), _ptr(conf), _ptr(tok),
                              _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
@@ -457,6 +467,8 @@ def ds_confidence_static(logits, conf, tok, row_list=None, stream=None):
         raise ValueError("conf must be f32 [rows] and tok i32 [rows]")
     if row_list is not None and row_list.dtype != torch.int32:
         raise TypeError("row_list must be int32")
+    if row_list is not None and row_list.numel() == 0:
+        return conf, tok      # no row listed: nothing is touched (a null list pointer would mean "all rows")
     rc = lib().ds_confidence_static(_ptr(logits), _dtype_code(logits), rows, V, logits.stride(0), _ptr(row_list),
                                     0 if row_list is None else row_list.numel(), _ptr(conf), _ptr(tok),
                                     _stream(stream))
@@ -530,6 +542,15 @@ def ds_block_begin(eos_exit, masked, x_block, mask_id, fill_id, active_seq, acti
     rc = lib().ds_block_begin(ctypes.byref(p), _stream(stream))
     if rc != DS_OK:
         raise DsError(rc, "ds_block_begin")
+
+
+def ds_selftest_bounded_wait(poll_limit: int, status=None, report=None, stream=None):
+    """Runs the kernels' bounded wait on a barrier nobody arrives on (see ds.h).  status: int32/uint32 [1],
+    report: int32 [3], both optional device tensors."""
+    _check_dev(status, report)
+    rc = lib().ds_selftest_bounded_wait(int(poll_limit), _ptr(status), _ptr(report), _stream(stream))
+    if rc != DS_OK:
+        raise DsError(rc, "ds_selftest_bounded_wait")
 
 
 def ds_read_status(status: torch.Tensor, stream=None) -> int:

@@ -1,8 +1,6 @@
 // C ABI of the denoising-step library: argument validation and dispatch.
 // Every step of the path runs in the CUDA kernels of the sibling files.
 #include <atomic>
-#include <cstdlib>
-#include <cstring>
 #include <new>
 
 #include "ds_common.cuh"
@@ -59,19 +57,14 @@ int validate_attn(const ds_attn_params *p) {
     }
     if (strides[k][2] < p->D) return DS_ERR_INVALID_ARG;  // rows must not overlap
   }
-  if (p->D % 32 != 0 || p->D > 256) return DS_ERR_UNSUPPORTED;
+  if (p->kernel != DS_ATTN_KERNEL_AUTO && p->kernel != DS_ATTN_KERNEL_ONE_TILE && p->kernel != DS_ATTN_KERNEL_TWO_TILE)
+    return DS_ERR_INVALID_ARG;
+  // The envelope: bf16 on the tensor cores, fp32 on the CUDA cores; nothing is rerouted.
   if (p->B > 65535 || p->Hq > 65535) return DS_ERR_UNSUPPORTED;
+  if (p->dtype == DS_BF16) return attn_tc_supported(*p) ? DS_OK : DS_ERR_UNSUPPORTED;
+  if (p->D != 32 && p->D != 64 && p->D != 128 && p->D != 256) return DS_ERR_UNSUPPORTED;
+  if (!(p->scale > -1e30f && p->scale < 1e30f)) return DS_ERR_UNSUPPORTED;
   return DS_OK;
-}
-
-enum class AttnPath { kAuto, kSimt, kTc, kTc2 };
-AttnPath forced_path() {
-  const char *e = std::getenv("DS_ATTN_PATH");
-  if (!e) return AttnPath::kAuto;
-  if (!std::strcmp(e, "simt")) return AttnPath::kSimt;
-  if (!std::strcmp(e, "tc")) return AttnPath::kTc;
-  if (!std::strcmp(e, "tc2")) return AttnPath::kTc2;
-  return AttnPath::kAuto;
 }
 
 }  // namespace
@@ -81,7 +74,8 @@ extern "C" {
 
 size_t ds_attn_pruned_workspace(const ds_attn_params *p) {
   if (ds::validate_attn(p) != DS_OK) return 0;
-  if (ds::forced_path() != ds::AttnPath::kSimt && ds::attn_tc_supported(*p)) return ds::attn_tc_workspace_bytes(*p);
+  // only the one-tile kernel splits the keys of an item over CTAs
+  if (p->dtype == DS_BF16 && p->kernel != DS_ATTN_KERNEL_TWO_TILE) return ds::attn_tc_workspace_bytes(*p);
   return 0;
 }
 
@@ -114,16 +108,13 @@ int resolve_attn(const ds_attn_params *p, AttnPrepared &a) {
   a.grid = 0;
   a.path = kAttnPathSimt;
   if (p->B == 0) return DS_OK;
-  const AttnPath path = forced_path();
-  const bool tc_ok = attn_tc_supported(*p);
-  if ((path == AttnPath::kTc || path == AttnPath::kTc2) && !tc_ok) return DS_ERR_UNSUPPORTED;
-  if (tc_ok && path == AttnPath::kTc2) return prepare_attn_tc2(*p, a);
-  if (tc_ok && path != AttnPath::kSimt) {
+  if (p->dtype == DS_BF16) {
+    if (p->kernel == DS_ATTN_KERNEL_TWO_TILE) return prepare_attn_tc2(*p, a);
+    if (p->kernel == DS_ATTN_KERNEL_AUTO && two_tile_kernel_pays(*p)) return prepare_attn_tc2(*p, a);
     // a missing or short workspace is not an error: the call then runs without splitting the keys
-    if (path == AttnPath::kAuto && two_tile_kernel_pays(*p)) return prepare_attn_tc2(*p, a);
     return prepare_attn_tc(*p, a);
   }
-  a.grid = 1;  // the SIMT launcher sizes its own grid from a.p
+  a.grid = 1;  // the fp32 launcher sizes its own grid from a.p
   return DS_OK;
 }
 
@@ -282,6 +273,12 @@ int ds_block_begin(const ds_block_params *p, void *stream) {
   if ((long long)p->B * p->K > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   if (p->B > 0 && (!p->eos_exit || !p->masked || !p->x_block || !p->active_seq)) return DS_ERR_INVALID_ARG;
   return ds::launch_block_begin(*p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int ds_selftest_bounded_wait(uint32_t poll_limit, uint32_t *status, int32_t *report, void *stream) {
+  if (poll_limit == 0 || poll_limit > (1u << 16)) return DS_ERR_INVALID_ARG;
+  if ((status && !ds::aligned(status, 4)) || (report && !ds::aligned(report, 4))) return DS_ERR_INVALID_ARG;
+  return ds::launch_bounded_wait_selftest(poll_limit, status, report, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int ds_last_cuda_error(void) { return ds::g_last_cuda_error; }

@@ -1,5 +1,4 @@
-// ds_attn_pruned, CUDA-core path: fp32 inputs (any head dimension that is a
-// multiple of 32 up to 256) and bf16 shapes the tensor-core kernel does not take.
+// ds_attn_pruned, CUDA-core path: fp32 inputs, head dimension 32, 64, 128 or 256.
 //
 // One warp owns one retained query row (Eq. 8: queries = current block U
 // retained suffix).  The lanes split the head dimension; keys are visited
@@ -13,8 +12,10 @@ namespace {
 
 constexpr int kRowsPerCta = 8;
 
+// A lane's slice of a row.  Rows are only promised 16-byte alignment (bases and strides), so a slice wider
+// than that (fp32, D = 256: 32 bytes) is moved as 16-byte pieces.
 template <typename T, int N>
-struct alignas(sizeof(T) * N) Frag {
+struct alignas(sizeof(T) * N < 16 ? sizeof(T) * N : 16) Frag {
   T v[N];
 };
 
@@ -22,14 +23,10 @@ template <typename T>
 __device__ __forceinline__ float to_f32(T x);
 template <>
 __device__ __forceinline__ float to_f32<float>(float x) { return x; }
-template <>
-__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
 template <typename T>
 __device__ __forceinline__ T from_f32(float x);
 template <>
 __device__ __forceinline__ float from_f32<float>(float x) { return x; }
-template <>
-__device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
 template <typename T, int DPL>
 __device__ __forceinline__ void load_frag(const T *p, float (&out)[DPL]) {
@@ -83,6 +80,7 @@ __global__ void __launch_bounds__(kRowsPerCta * 32) attn_simt_kernel(const ds_at
 
   float q[DPL];
   load_frag<T, DPL>(Qt + (long long)tail_row(i) * p.q_stride[2] + dofs, q);
+  if (i > 0 && ix[i] <= ix[i - 1]) bad_index = true;  // the list must be strictly ascending (served as written)
   const float qs = p.scale * kLog2e;
 #pragma unroll
   for (int k = 0; k < DPL; ++k) q[k] *= qs;
@@ -173,9 +171,9 @@ int launch_t(const ds_attn_params &p, cudaStream_t stream) {
 }  // namespace
 
 int launch_attn_simt(const ds_attn_params &p, cudaStream_t stream) {
-  if (p.D % 32 != 0 || p.D > 256) return DS_ERR_UNSUPPORTED;
+  if (p.dtype != DS_F32) return DS_ERR_UNSUPPORTED;
   if (p.Hq > 65535 || p.B > 65535) return DS_ERR_UNSUPPORTED;
-  return p.dtype == DS_BF16 ? launch_t<__nv_bfloat16>(p, stream) : launch_t<float>(p, stream);
+  return launch_t<float>(p, stream);
 }
 
 }  // namespace ds

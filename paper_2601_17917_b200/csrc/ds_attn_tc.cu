@@ -48,7 +48,6 @@
 // for (bounded), TMEM is freed and the CTA returns.
 #include <cuda.h>
 
-#include <cstdio>
 #include <cstring>
 #include <mutex>
 
@@ -62,19 +61,6 @@ namespace {
 
 using namespace sm100;
 using namespace attn;
-
-// Optional timeline of CTA 0 (build with -DDS_TRACE): SM clock at a few points of every role's loop.
-#ifdef DS_TRACE
-__device__ long long g_trace[4][256][8];
-#define DS_TR(role, g, ev)                                              \
-  do {                                                                  \
-    if (blockIdx.x == 0 && (g) < 256) g_trace[role][g][ev] = clock64(); \
-  } while (0)
-#else
-#define DS_TR(role, g, ev) \
-  do {                     \
-  } while (0)
-#endif
 
 constexpr int kSoftmaxWarps = 8;
 constexpr int kXWarps = 4;  // softmax of the transposed problem (one per TMEM lane quadrant)
@@ -250,18 +236,12 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     }
     // one index list for all batches: keep (the head of) it in shared memory, validated once
     const int32_t *idx_cache = nullptr;
+    bool list_ok = false;  // the list is known to be in range and strictly ascending
     if (prm.idx_bstride == 0) {
       int32_t *cache = reinterpret_cast<int32_t *>(smem + G_::kOffIdxCache);
-      for (int i = lane; i < min(prm.Lq, kIdxCap); i += 32) {
-        int v = prm.idx[i];
-        if (v < 0 || v >= prm.T) {
-          bad_index = true;
-          v = v < 0 ? 0 : prm.T - 1;
-        }
-        cache[i] = v;
-      }
+      list_ok = cache_shared_index_list(prm, cache, bad_index);
       __syncwarp();
-      idx_cache = cache;
+      if (list_ok) idx_cache = cache;  // a malformed list is read entry by entry from global memory
     }
     const int n_my = (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // items of this CTA
     int q_next = 0;  // first item (in this CTA's order) whose query tile has not been requested yet
@@ -270,14 +250,14 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     auto issue_q = [&](int kq) {
       const Item it = decode_item<kSplit>(prm, blockIdx.x + kq * gridDim.x);
       uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
-                                      it.mt * kBlockM, it.m_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
+                                      it.mt * kBlockM, it.m_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index);
       if (it.x_rows > 0) {
         // rows of the small query tile that are not loaded must be finite: clear the tile first
         for (int q = lane; q < (2 * kXChunkBytes) / 16; q += 32)
           *reinterpret_cast<uint4 *>(smem + G_::kOffQx + q * 16) = make_uint4(0, 0, 0, 0);
         fence_proxy_async();
         bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQx, kXChunkBytes, bar_q_full,
-                                (it.mt + 1) * kBlockM, it.x_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
+                                (it.mt + 1) * kBlockM, it.x_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index);
       }
       if (lane == 0) mbar_arrive_expect_tx(bar_q_full, bytes);
     };
@@ -291,7 +271,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           const int slot = issued % G_::kSlots, use = issued / G_::kSlots;
           const uint32_t dst = sbase + G_::kOffRing + slot * G_::kTileBytes;
           const uint32_t full = bar_slot_full + 8 * slot;
-          DS_TR(0, issued >> 1, kv * 3 + 0);
           // Wait for the ring slot.  The KV stream runs ahead of the query tiles across item
           // boundaries, so while waiting, serve the query tile of the item these fills belong to as
           // soon as the previous item has released the buffer.
@@ -322,7 +301,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
             timed_out = true;
             break;
           }
-          DS_TR(0, issued >> 1, kv * 3 + 1);
           if (j < n_pre) {
             {
               // one lane per 64-column chunk: the copies are issued side by side
@@ -346,10 +324,9 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
             }
             // the V fill of a tile directly follows its K fill: the staged row list is still valid
             const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, kv ? &prm.v128 : &prm.k128, dst, kChunkBytes,
-                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, bad_index, kv == 1);
+                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, list_ok, bad_index, kv == 1);
             if (lane == 0) mbar_arrive_expect_tx(full, bytes);
           }
-          DS_TR(0, issued >> 1, kv * 3 + 2);
           ++issued;
         }
       }
@@ -412,7 +389,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         tc_fence_after();
         const uint64_t dk = dk0 + (uint64_t)((slot * G_::kTileBytes) >> 4);
         if (elect_one()) {
-          DS_TR(1, g, 0);
           const uint32_t d = tm + ((g & 1) ? G_::kTmemS1 : G_::kTmemS0);
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
@@ -444,7 +420,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           }
           umma_commit(bar_slot_empty + 8 * slot);
           if (jj == nt_cur - 1) umma_commit(bar_q_free);
-          DS_TR(1, g, 1);
         }
         __syncwarp();
       }
@@ -482,7 +457,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         tc_fence_after();
         const uint64_t dv = dv0 + (uint64_t)((slot * G_::kTileBytes) >> 4);
         if (elect_one()) {
-          DS_TR(1, g, 2);
 #pragma unroll
           for (int ks = 0; ks < kBlockN / 16; ++ks)
             umma_ts(tm + G_::kTmemO, tm + ((g & 1) ? G_::kTmemS1 : G_::kTmemS0) + ks * 8, dv + ((ks * 2048) >> 4),
@@ -513,7 +487,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           }
           umma_commit(bar_slot_empty + 8 * slot);
           if (jj == nt_cur - 1) umma_commit(bar_o_full);
-          DS_TR(1, g, 3);
         }
         __syncwarp();
       }
@@ -696,8 +669,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     const uint32_t lane_base = tmem + ((uint32_t)lane0 << 16);
     const float c2 = prm.scale_log2;
     constexpr int kOCols = D / 2;                          // accumulator columns per thread
-    const bool tracer = (warp & 3) == 0 && lane == 0;
-    (void)tracer;
     bool ok = true;
     int g0 = 0, k = 0;
     int nt_cur = 0;  // KV tiles of the current item that this CTA processes
@@ -715,13 +686,11 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        if (tracer) DS_TR(2 + (warp >> 2), g, 0);
         const uint32_t s_base = lane_base + ((g & 1) ? G_::kTmemS1 : G_::kTmemS0);
         uint32_t s[64];
         tmem_ld16x2_32<64>(s_base, &s[0]);        // columns 64 half + 0..31
         tmem_ld16x2_32<64>(s_base + 32, &s[32]);  // columns 64 half + 32..63
         tmem_wait_ld();
-        if (tracer) DS_TR(2 + (warp >> 2), g, 1);
         // columns past the end of a partial tile do not exist
         const int valid = (j < n_pre) ? min(kBlockN, prm.P - j * kBlockN) : min(kBlockN, prm.Lq - (j - n_pre) * kBlockN);
         if (valid < kBlockN) {
@@ -748,7 +717,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           mx = fmax3(mx, a[6], a[7]);
           mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
         }
-        if (tracer) DS_TR(2 + (warp >> 2), g, 2);
         const float m_tile = mx * c2;
         float factor = 1.f;
         if (m_tile > m_used + kRescaleThreshold || m_used == -INFINITY) {
@@ -774,7 +742,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           l3 += p3;
         }
         l_sum += (l0 + l1) + (l2 + l3);
-        if (tracer) DS_TR(2 + (warp >> 2), g, 3);
         if (warp_rescales) {
           // O must be quiescent: the previous P V has completed
           ok = mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag);
@@ -791,7 +758,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
             tmem_st16x2_32<kOCols>(lane_base + G_::kTmemO + cb, o);
           }
         }
-        if (tracer) DS_TR(2 + (warp >> 2), g, 4);
         // P row -> TMEM over the first 64 columns of its own S buffer (two bf16 per column); this
         // thread's 64 keys are columns 32 half .. 32 half + 31
         tmem_st16x2_32<32>(s_base, pk);
@@ -799,7 +765,6 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_p_full + 8 * (g & 1));
-        if (tracer) DS_TR(2 + (warp >> 2), g, 5);
       }
       if (!ok) break;
       // ---- epilogue of the item ----
@@ -942,7 +907,10 @@ int prepare_d(const ds_attn_params &p, AttnPrepared &out) {
   out.path = kAttnPathTc;
   out.p = p;
   out.grid = 0;
-  if (!fill_common(prm, p)) return DS_ERR_CUDA;
+  if (!fill_common(prm, p)) {
+    note_cuda_error((int)cudaErrorInvalidValue);  // cuTensorMapEncodeTiled refused the layout
+    return DS_ERR_CUDA;
+  }
   tile_counts(p, prm.n_mtiles, prm.x_rows);
   const int n_tiles = (p.P + kBlockN - 1) / kBlockN + (p.Lq + kBlockN - 1) / kBlockN;
   prm.splits = 1;
@@ -1066,16 +1034,17 @@ EncodeFn encode_fn() {
 }
 }  // namespace sm100
 
-#ifdef DS_TRACE
-extern "C" __attribute__((visibility("default"))) int ds_debug_trace(long long *host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : 1;
-}
-#endif
-
 bool attn_tc_supported(const ds_attn_params &p) {
   if (p.dtype != DS_BF16 || (p.D != 64 && p.D != 128)) return false;
   if (!(p.scale > 0.f) || p.scale > 1e30f) return false;  // the running maximum assumes a positive scale
   if ((long long)(p.Hq / p.Hkv) * p.Lq > (1ll << 30)) return false;
+  // a tensor map has no broadcast dimension: batch and head strides of extents above 1 must be positive
+  const int64_t *st[3] = {p.q_stride, p.kv_tail_stride, p.kv_prefix_stride};
+  const int heads[3] = {p.Hq, p.Hkv, p.Hkv};
+  for (int k = 0; k < 3; ++k) {
+    if (k == 2 && p.P == 0) continue;
+    if ((p.B > 1 && st[k][0] <= 0) || (heads[k] > 1 && st[k][1] <= 0)) return false;
+  }
   // TMA: 16-byte aligned bases and strides are already guaranteed by validation; extents must fit 32 bits
   return true;
 }

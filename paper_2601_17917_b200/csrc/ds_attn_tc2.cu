@@ -157,28 +157,22 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
       prefetch_map(&prm.q128);
     }
     const int32_t *idx_cache = nullptr;
+    bool list_ok = false;  // the list is known to be in range and strictly ascending
     if (prm.idx_bstride == 0) {
       int32_t *cache = reinterpret_cast<int32_t *>(smem + G_::kOffIdxCache);
-      for (int i = lane; i < min(prm.Lq, kIdxCap); i += 32) {
-        int v = prm.idx[i];
-        if (v < 0 || v >= prm.T) {
-          bad_index = true;
-          v = v < 0 ? 0 : prm.T - 1;
-        }
-        cache[i] = v;
-      }
+      list_ok = cache_shared_index_list(prm, cache, bad_index);
       __syncwarp();
-      idx_cache = cache;
+      if (list_ok) idx_cache = cache;  // a malformed list is read entry by entry from global memory
     }
     const int n_my = (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     int q_next = 0;
     auto issue_q = [&](int kq) {
       const Item2 it = decode_item2(prm, blockIdx.x + kq * gridDim.x);
       uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
-                                      it.pr * 2 * kBlockM, it.rows_a, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
+                                      it.pr * 2 * kBlockM, it.rows_a, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index);
       if (it.rows_b > 0)
         bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ + G_::kTileBytes, kChunkBytes, bar_q_full,
-                                (it.pr * 2 + 1) * kBlockM, it.rows_b, it.hk * prm.G, it.b, idxq_s, idx_cache, bad_index);
+                                (it.pr * 2 + 1) * kBlockM, it.rows_b, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index);
       if (lane == 0) mbar_arrive_expect_tx(bar_q_full, bytes);
     };
     int issued = 0;
@@ -237,7 +231,7 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
               fence_proxy_async();
             }
             const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, kv ? &prm.v128 : &prm.k128, dst, kChunkBytes,
-                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, bad_index, kv == 1);
+                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, list_ok, bad_index, kv == 1);
             if (lane == 0) mbar_arrive_expect_tx(full, bytes);
           }
           ++issued;
@@ -544,7 +538,10 @@ int prepare2_d(const ds_attn_params &p, AttnPrepared &out) {
   out.path = kAttnPathTc2;
   out.p = p;
   out.grid = 0;
-  if (!fill_common(prm, p)) return DS_ERR_CUDA;
+  if (!fill_common(prm, p)) {
+    note_cuda_error((int)cudaErrorInvalidValue);  // cuTensorMapEncodeTiled refused the layout
+    return DS_ERR_CUDA;
+  }
   const long long rows_total = (long long)prm.G * p.Lq;
   prm.n_pairs = (int)((rows_total + 2 * kBlockM - 1) / (2 * kBlockM));
   const long long n_items = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv * prm.n_pairs;  // upper bound with a device count

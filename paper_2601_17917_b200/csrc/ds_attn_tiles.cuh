@@ -54,17 +54,47 @@ __device__ __forceinline__ bool bad_sequence_numbers(const AttnCommon &c, int n_
 }
 
 // ------------------------------------------------------------------------------------------------
+// Producer helper: the index list shared by all batches (idx_bstride == 0) is checked once per CTA --
+// every entry in [0, T), strictly ascending -- and its head is kept in shared memory.  Returns true when
+// the whole list passed; the caller then passes list_ok = true to gather_rows, which may decide from the
+// first and last entry of a run that the rows between them are consecutive.  Entries out of range are
+// clamped in the cached copy and flagged.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool cache_shared_index_list(const AttnCommon &prm, int32_t *cache, bool &bad_index) {
+  const int lane = threadIdx.x & 31;
+  bool ok = true;
+  for (int i = lane; i < prm.Lq; i += 32) {
+    int v = prm.idx[i];
+    const int before = (i > 0) ? prm.idx[i - 1] : -1;
+    if (v < 0 || v >= prm.T) {
+      ok = false;
+      v = v < 0 ? 0 : prm.T - 1;
+    }
+    if (v <= before) ok = false;
+    if (i < kIdxCap) cache[i] = v;
+  }
+  ok = __all_sync(0xffffffffu, ok);
+  if (!ok) bad_index = true;
+  return ok;
+}
+
+// ------------------------------------------------------------------------------------------------
 // Producer helper: fetch n gathered rows (logical rows R0 .. R0+n-1 of a stacked sequence whose
 // period is Lq) into a swizzled tile whose 64-column chunks are chunk_stride bytes apart.  The whole
 // warp calls it; lane 0 issues the copies (a whole-tile fetch: one lane per chunk).  Returns the bytes issued.
+//
+// Runs of consecutive rows are fetched as one box (128 or 32 rows).  With list_ok (the list is known to be
+// strictly ascending and in range) the first and last entry of a run decide; otherwise every entry of the
+// run is looked at, and a tile whose entries are not strictly ascending is flagged and fetched row by row.
 // ------------------------------------------------------------------------------------------------
 template <int D>
 __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUtensorMap *map32, const CUtensorMap *map1,
                                                 const CUtensorMap *map128, uint32_t dst, uint32_t chunk_stride, uint32_t bar, int R0, int n,
-                                                int head0, int b, int32_t *idx_s, const int32_t *idx_cache,
+                                                int head0, int b, int32_t *idx_s, const int32_t *idx_cache, bool list_ok,
                                                 bool &bad_index, bool staged = false) {
   const int lane = threadIdx.x & 31;
   const int Lq = prm.Lq;
+  const int32_t *ix = prm.idx + (long long)b * prm.idx_bstride;
   // position of logical row R0 inside its head; divisions only when the stacking actually wraps
   int head = head0, pos0 = R0;
   if (pos0 >= Lq) {
@@ -72,26 +102,32 @@ __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUt
     pos0 %= Lq;
   }
   // A full tile of consecutive rows inside one head (the current block and its window, every tile of a
-  // cache-refresh step) needs no staging: the list is strictly ascending, so its first and last entry
-  // decide, and one box per 64-column chunk fetches it, each chunk issued by a lane of its own.
+  // cache-refresh step) needs no staging: one box per 64-column chunk fetches it, each chunk issued by a
+  // lane of its own.
   if (n == 128 && pos0 + 128 <= Lq) {
     int first, last;
     if (idx_cache != nullptr && pos0 + 127 < kIdxCap) {
       first = idx_cache[pos0];
       last = idx_cache[pos0 + 127];
     } else {
-      const int32_t *ix = prm.idx + (long long)b * prm.idx_bstride;
       first = ix[pos0];
       last = ix[pos0 + 127];
     }
-    if (last - first == 127 && first >= 0 && last < prm.T) {
+    bool whole = (last - first == 127 && first >= 0 && last < prm.T);
+    if (whole && !list_ok) {
+      // the order of the list is not known: all 128 entries must be the consecutive rows
+      bool run = true;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) run = run && (ix[pos0 + lane + 32 * k] == first + lane + 32 * k);
+      whole = __all_sync(0xffffffffu, run);
+    }
+    if (whole) {
       if (lane < (D / 64)) tma_load_4d(dst + lane * chunk_stride, map128, bar, lane * 64, first, head, b);
       return 128u * 128u * (D / 64);
     }
   }
   __syncwarp();
   if (!staged) {  // otherwise idx_s already holds these rows (the K tile of the same rows came first)
-    const int32_t *ix = prm.idx + (long long)b * prm.idx_bstride;
     for (int r = lane; r < n; r += 32) {
       int pos = pos0 + r;
       if (pos >= Lq) pos %= Lq;
@@ -109,12 +145,24 @@ __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUt
     }
     __syncwarp();
   }
+  // may runs of this tile be fetched as 32-row boxes?  (a box follows the memory order of the rows)
+  bool boxes = list_ok;
+  if (!list_ok) {
+    bool asc = true;
+    for (int r = lane + 1; r < n; r += 32) {
+      int pos = pos0 + r;
+      if (pos >= Lq) pos %= Lq;
+      asc = asc && (pos == 0 || idx_s[r] > idx_s[r - 1]);  // the stacking starts the list again at every head
+    }
+    boxes = __all_sync(0xffffffffu, asc);
+    if (!boxes) bad_index = true;
+  }
   uint32_t bytes = 0;
   if (lane == 0) {
     int r = 0, pos = pos0;
     while (r < n) {
       const int row = idx_s[r];
-      const bool box32 = ((r & 7) == 0) && (r + 32 <= n) && (pos + 32 <= Lq) && (idx_s[r + 31] - row == 31);
+      const bool box32 = boxes && ((r & 7) == 0) && (r + 32 <= n) && (pos + 32 <= Lq) && (idx_s[r + 31] - row == 31);
       const int step = box32 ? 32 : 1;
 #pragma unroll
       for (int c = 0; c < (D / 64); ++c)

@@ -53,6 +53,7 @@ int launch_lmhead_confidence(const void *hidden, const void *weight, int64_t row
 int launch_block_begin(const ds_block_params &p, cudaStream_t stream);
 int launch_select(const ds_select_params &p, cudaStream_t stream);
 int launch_rope_gather(const ds_rope_params &p, cudaStream_t stream);
+int launch_bounded_wait_selftest(uint32_t poll_limit, uint32_t *status, int32_t *report, cudaStream_t stream);
 void note_cuda_error(int code);  // remembered per host thread for ds_last_cuda_error
 int launch_attn_simt(const ds_attn_params &p, cudaStream_t stream);
 int launch_attn_tc(const ds_attn_params &p, cudaStream_t stream);

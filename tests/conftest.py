@@ -16,3 +16,15 @@ def pytest_configure(config):
 @pytest.fixture(scope="session")
 def golden_dir():
     return ROOT / "tests" / "golden"
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Worst max-abs-err / RMS(O) ratios of the attention parity comparisons (tests/test_gpu_attn.py)."""
+    mod = sys.modules.get("test_gpu_attn") or sys.modules.get("tests.test_gpu_attn")
+    rows = getattr(mod, "ERR_OVER_RMS", None)
+    if not rows:
+        return
+    rows = sorted(rows, reverse=True)
+    terminalreporter.write_line(f"attention parity: {len(rows)} comparisons, worst max-abs-err / RMS(O):")
+    for ratio, err, rms, what in rows[:8]:
+        terminalreporter.write_line(f"  {ratio:.3e}  (err {err:.3e}, rms {rms:.3e})  {what}")

@@ -41,9 +41,9 @@ def test_ctypes_structs_match_header(tmp_path):
 #include <stddef.h>
 #include "ds.h"
 int main(void) {
-  printf("%zu %zu %zu %zu %zu %zu\n", sizeof(ds_attn_params), offsetof(ds_attn_params, q_stride),
+  printf("%zu %zu %zu %zu %zu %zu %zu\n", sizeof(ds_attn_params), offsetof(ds_attn_params, q_stride),
          offsetof(ds_attn_params, idx), offsetof(ds_attn_params, scale), offsetof(ds_attn_params, out),
-         offsetof(ds_attn_params, status));
+         offsetof(ds_attn_params, status), offsetof(ds_attn_params, kernel));
   printf("%zu %zu %zu %zu %zu\n", sizeof(ds_select_params), offsetof(ds_select_params, tau0),
          offsetof(ds_select_params, seq_list), offsetof(ds_select_params, n_seq_dev),
          offsetof(ds_select_params, active_cnt));
@@ -59,7 +59,7 @@ int main(void) {
     assert [int(v) for v in r.split()] == [ctypes.sizeof(R), R.q_stride.offset, R.idx.offset, R.rope_theta.offset,
                                            R.k_cache.offset, R.status.offset]
     assert [int(v) for v in a.split()] == [ctypes.sizeof(A), A.q_stride.offset, A.idx.offset, A.scale.offset,
-                                           A.out.offset, A.status.offset]
+                                           A.out.offset, A.status.offset, A.kernel.offset]
     assert [int(v) for v in s.split()] == [ctypes.sizeof(S), S.tau0.offset, S.seq_list.offset,
                                            S.n_seq_dev.offset, S.active_cnt.offset]
 
@@ -103,6 +103,40 @@ def test_attention_argument_validation_needs_no_gpu(L):
                                                out_stride=(4 * 8 * 48, 8 * 48, 48))), None) == ds.DS_ERR_UNSUPPORTED
     # B = 0 is a valid empty call
     assert L.ds_attn_pruned(ctypes.byref(_attn(B=0)), None) == ds.DS_OK
+
+
+def test_attention_envelope_refuses_instead_of_rerouting(L):
+    """bf16 is served by the tensor-core kernels only (D 64 or 128, positive scale) and fp32 by the CUDA-core
+    kernel only (D 32, 64, 128, 256): a well-formed request outside that is DS_ERR_UNSUPPORTED, decided on
+    the host before any device is touched.  The kernel choice is an explicit field, not an environment
+    variable."""
+    def shaped(D, **kw):
+        st = (4 * 8 * D, 8 * D, D)
+        return _attn(**{**dict(D=D, q_stride=st, kv_tail_stride=st, out_stride=st), **kw})
+    for p in (shaped(96), shaped(32), shaped(160), shaped(256), shaped(128, scale=0.0), shaped(64, scale=-0.125),
+              shaped(96, dtype=ds.DS_F32), shaped(224, dtype=ds.DS_F32),
+              shaped(128, B=2, q_stride=(0, 8 * 128, 128))):            # a broadcast batch: no tensor map for it
+        assert L.ds_attn_pruned(ctypes.byref(p), None) == ds.DS_ERR_UNSUPPORTED
+        assert L.ds_attn_pruned_workspace(ctypes.byref(p)) == 0
+        h = ctypes.c_void_p()
+        assert L.ds_attn_plan_create(ctypes.byref(p), ctypes.byref(h)) == ds.DS_ERR_UNSUPPORTED and not h.value
+    for k in (-1, 3, 100):
+        assert L.ds_attn_pruned(ctypes.byref(_attn(kernel=k)), None) == ds.DS_ERR_INVALID_ARG
+    import os
+    os.environ["DS_ATTN_PATH"] = "simt"          # the library reads no environment
+    try:
+        assert L.ds_attn_pruned(ctypes.byref(shaped(96)), None) == ds.DS_ERR_UNSUPPORTED
+    finally:
+        del os.environ["DS_ATTN_PATH"]
+    src = "".join(f.read_text() for f in (ROOT / "paper_2601_17917_b200" / "csrc").glob("*.cu*"))
+    assert "getenv" not in src
+
+
+def test_bounded_wait_selftest_argument_validation(L):
+    fake = ctypes.c_void_p(0x7f0000000000)
+    assert L.ds_selftest_bounded_wait(0, fake, fake, None) == ds.DS_ERR_INVALID_ARG
+    assert L.ds_selftest_bounded_wait(1 << 20, fake, fake, None) == ds.DS_ERR_INVALID_ARG
+    assert L.ds_selftest_bounded_wait(100, ctypes.c_void_p(0x7f0000000002), fake, None) == ds.DS_ERR_INVALID_ARG
 
 
 def test_confidence_and_select_argument_validation(L):

@@ -1,11 +1,16 @@
 """GPU parity of ds_attn_pruned (Eq. 7-8) against the CPU oracle, through the C ABI.
 
 Bar: max-abs error <= 1e-2 on unit-scale values.  With N(0,1) inputs the
-outputs are small (softmax is diffuse), so the error is also bounded relative
-to the RMS of the reference output, and a "peaked" case (queries x4) gives
-unit-scale outputs.  Small cases are compared element by element; the full
-size configurations on sampled (batch, head) slices and sampled query rows,
-which the oracle computes one by one from the same device-generated data."""
+outputs are small (softmax is diffuse: typical |O| is 0.03-0.15), so every
+comparison is also bounded by the kernel's own error model, which is relative:
+bf16 output rounding (2^-9 of the value) plus the bf16 rounding of the
+probabilities, which shows up as a fraction of the RMS of the reference output.
+The ratio max-abs-err / RMS(O) of every comparison is collected and the worst
+ones are printed in the test summary.  A "peaked" case (queries x4) gives
+unit-scale outputs.  Small cases are compared element by element; the two
+long-context bench workloads on every (batch, head) slice; the other full-size
+configurations on sampled slices and sampled query rows, which the oracle
+computes one by one from the same device-generated data."""
 import math
 
 import numpy as np
@@ -21,9 +26,15 @@ DEV = "cuda:0"
 ABS_BAR = 1e-2
 
 
+# max-abs-err / RMS(O) of every comparison made in this module: (ratio, err, rms, what)
+ERR_OVER_RMS = []
+# The kernel's own error model, elementwise: |out - ref| <= REL * |ref| + RMS_FRAC * RMS(ref) + ABS.
+#   bf16: REL = 2^-8 (output rounding is 2^-9; the split path rounds partial results once more),
+#         RMS_FRAC = 2.5e-2 (bf16 probabilities: 2^-9 relative each, a few sigma over ~1e6 elements,
+#         plus the approximate exponential), ABS = 1e-6
+#   fp32: REL = 1e-5, RMS_FRAC = 1e-4, ABS = 1e-6
 def _tol(dtype):
-    # own bounds: fp32 path ~1e-5; bf16 path = output rounding (2^-9 relative) + bf16 probabilities
-    return (2e-5, 1e-4) if dtype == torch.float32 else (4e-3, 2e-2)
+    return (1e-5, 1e-4, 1e-6) if dtype == torch.float32 else (2.0 ** -8, 2.5e-2, 1e-6)
 
 
 def _np(t):
@@ -32,18 +43,20 @@ def _np(t):
 
 def _compare(out, ref, dtype, what=""):
     out = _np(out).astype(np.float64)
-    err = np.abs(out - ref).max()
+    diff = np.abs(out - ref)
+    err = diff.max()
     rms = math.sqrt(float((ref ** 2).mean())) + 1e-30
-    own_abs, own_rel = _tol(dtype)
+    rel, rms_frac, floor = _tol(dtype)
     assert np.isfinite(out).all(), what
     # the stated bar: 1e-2 max-abs on unit-scale values (bf16 cannot hold 1e-2 absolute beyond |x| = 2.56)
-    assert (np.abs(out - ref) <= ABS_BAR * np.maximum(1.0, np.abs(ref))).all(), (what, err)
-    assert err <= own_abs + own_rel * max(rms, np.abs(ref).max()), (what, err, rms)
+    assert (diff <= ABS_BAR * np.maximum(1.0, np.abs(ref))).all(), (what, err)
+    ERR_OVER_RMS.append((err / rms, err, rms, what))
+    assert (diff <= rel * np.abs(ref) + rms_frac * rms + floor).all(), (what, err, rms, err / rms)
     return err, rms
 
 
 def _run_small(B, Hq, Hkv, D, P, T, idx, dtype, seed=0, q_scale=1.0, want_lse=True, noncontig=False,
-               k_boost=None):
+               k_boost=None, kernel=ds.DS_ATTN_KERNEL_AUTO, expect_status=0):
     cfg = wl.StepConfig("t", B=B, Hq=Hq, Hkv=Hkv, D=D, P=P, gen=T, K=1, w=0, keep_last=False,
                         dtype="f32" if dtype == torch.float32 else "bf16", V=8, spike_p=0, seed=seed)
     x = wl.attention_inputs(cfg, device=DEV, q_scale=q_scale)
@@ -61,9 +74,10 @@ def _run_small(B, Hq, Hkv, D, P, T, idx, dtype, seed=0, q_scale=1.0, want_lse=Tr
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     scale = 1.0 / math.sqrt(D)
     kp, vp = (x["k_pre"], x["v_pre"]) if P > 0 else (None, None)
-    out = ds.ds_attn_pruned(x["q_tail"], x["k_tail"], x["v_tail"], kp, vp, idx_t, scale, lse=lse, status=status)
+    out = ds.ds_attn_pruned(x["q_tail"], x["k_tail"], x["v_tail"], kp, vp, idx_t, scale, lse=lse, status=status,
+                            kernel=kernel)
     torch.cuda.synchronize()
-    assert ds.ds_read_status(status) == 0
+    assert ds.ds_read_status(status) == expect_status
     ref, ref_lse = oracle.attn(_np(x["q_tail"]), _np(x["k_tail"]), _np(x["v_tail"]), _np(x["k_pre"]),
                                _np(x["v_pre"]), np.asarray(idx), scale, want_lse=True)
     _compare(out, ref, dtype, f"B{B} Hq{Hq} Hkv{Hkv} D{D} P{P} T{T} Lq{Lq}")
@@ -127,20 +141,88 @@ def test_many_items_per_cta():
     _run_small(40, 8, 4, 128, 300, 300, list(range(256)) + [299], torch.bfloat16, seed=80)  # 2 tiles + 2 extra rows
 
 
+KERNELS = {"tc": ds.DS_ATTN_KERNEL_ONE_TILE, "tc2": ds.DS_ATTN_KERNEL_TWO_TILE, "auto": ds.DS_ATTN_KERNEL_AUTO}
+
+
 @pytest.mark.parametrize("path", ["tc", "tc2"])
-def test_both_tensor_core_kernels_on_the_same_shapes(path, monkeypatch):
-    """The one-tile and the two-tile kernel are chosen by shape; here each is forced on shapes of both kinds
-    (several M-tiles per KV head, a single partial tile, GQA stacking, D = 64, no prefix, peaked scores)."""
-    monkeypatch.setenv("DS_ATTN_PATH", path)
+def test_both_tensor_core_kernels_on_the_same_shapes(path):
+    """The one-tile and the two-tile kernel are chosen by shape; here each is pinned (the `kernel` field of the
+    call) on shapes of both kinds (several M-tiles per KV head, a single partial tile, GQA stacking, D = 64,
+    no prefix, peaked scores)."""
+    kw = dict(kernel=KERNELS[path])
     T = 300
-    _run_small(2, 2, 2, 128, 300, T, list(range(256)) + [T - 1], torch.bfloat16, seed=31)
-    _run_small(1, 14, 2, 128, 512, T, list(range(96)) + [T - 1], torch.bfloat16, seed=32)
-    _run_small(2, 4, 4, 128, 1000, 400, list(range(320)) + [399], torch.bfloat16, seed=33, q_scale=2.0)
-    _run_small(1, 2, 2, 64, 200, T, list(range(T)), torch.bfloat16, seed=34)
-    _run_small(3, 8, 2, 128, 0, 200, list(range(129)) + [199], torch.bfloat16, seed=35)
-    _run_small(40, 8, 4, 128, 300, T, list(range(256)) + [T - 1], torch.bfloat16, seed=36)
-    _run_small(1, 2, 2, 128, 130, 200, list(range(63)) + [199], torch.bfloat16, seed=37, q_scale=3.0)
-    _run_small(1, 2, 2, 128, 700, 200, list(range(128)) + [199], torch.bfloat16, seed=38, q_scale=3.0, k_boost=(300, 5.0))
+    _run_small(2, 2, 2, 128, 300, T, list(range(256)) + [T - 1], torch.bfloat16, seed=31, **kw)
+    _run_small(1, 14, 2, 128, 512, T, list(range(96)) + [T - 1], torch.bfloat16, seed=32, **kw)
+    _run_small(2, 4, 4, 128, 1000, 400, list(range(320)) + [399], torch.bfloat16, seed=33, q_scale=2.0, **kw)
+    _run_small(1, 2, 2, 64, 200, T, list(range(T)), torch.bfloat16, seed=34, **kw)
+    _run_small(3, 8, 2, 128, 0, 200, list(range(129)) + [199], torch.bfloat16, seed=35, **kw)
+    _run_small(40, 8, 4, 128, 300, T, list(range(256)) + [T - 1], torch.bfloat16, seed=36, **kw)
+    _run_small(1, 2, 2, 128, 130, 200, list(range(63)) + [199], torch.bfloat16, seed=37, q_scale=3.0, **kw)
+    _run_small(1, 2, 2, 128, 700, 200, list(range(128)) + [199], torch.bfloat16, seed=38, q_scale=3.0, k_boost=(300, 5.0), **kw)
+
+
+@pytest.mark.parametrize("path", ["tc", "tc2"])
+def test_index_list_that_is_not_ascending_is_flagged_and_served_as_written(path):
+    """The kernels fetch runs of consecutive rows as one box, deciding from the first and last entry of a run;
+    that is only sound for a strictly ascending list, so the order is checked on the device.  A list that
+    breaks it (here: two entries swapped inside a run whose ends still look like 128 consecutive rows, a
+    repeated row, a per-batch list with a descending step) raises DS_DEV_INDEX and every row is still the one
+    the list names, in the list's order."""
+    kw = dict(kernel=KERNELS[path], expect_status=ds.DS_DEV_INDEX)
+    T = 300
+    swapped = list(range(128))
+    swapped[5], swapped[6] = 6, 5
+    _run_small(2, 2, 2, 128, 200, T, swapped + [T - 1], torch.bfloat16, seed=41, **kw)
+    repeated = list(range(40)) + [39] + list(range(40, 100))
+    _run_small(1, 4, 2, 128, 130, T, repeated, torch.bfloat16, seed=42, **kw)
+    per_batch = np.stack([np.arange(160), np.arange(160)])
+    per_batch[1, 31], per_batch[1, 32] = 32, 31
+    _run_small(2, 2, 2, 128, 64, T, per_batch, torch.bfloat16, seed=43, **kw)
+    # the same shapes with well-formed lists raise nothing
+    _run_small(2, 2, 2, 128, 64, T, np.stack([np.arange(160), np.arange(3, 163)]), torch.bfloat16, seed=44,
+               kernel=KERNELS[path])
+
+
+@pytest.mark.parametrize("D", [32, 128, 256])
+def test_fp32_path_wide_heads_and_padded_rows(D):
+    """The fp32 kernel at every head dimension it takes, on contiguous and on strided inputs whose rows are
+    16-byte but not 32-byte aligned (a lane's slice of a D = 256 row is 32 bytes wide)."""
+    idx = list(range(40)) + [99]
+    _run_small(2, 4, 2, D, 70, 100, idx, torch.float32, seed=50 + D)
+    cfg = wl.StepConfig("t", B=1, Hq=2, Hkv=2, D=D, P=33, gen=100, K=1, w=0, keep_last=False, dtype="f32", V=8,
+                        spike_p=0, seed=60 + D)
+    x = wl.attention_inputs(cfg, device=DEV)
+    pad = {}
+    for k, t in x.items():      # row stride D + 4 floats: every other row starts 16 bytes off a 32-byte boundary
+        big = torch.zeros(t.shape[0], t.shape[1], t.shape[2], D + 4, dtype=t.dtype, device=DEV)
+        big[..., :D] = t
+        pad[k] = big[..., :D]
+    idx_t = torch.tensor(idx, dtype=torch.int32, device=DEV)
+    out_big = torch.zeros(1, 2, len(idx), D + 4, dtype=torch.float32, device=DEV)
+    out = ds.ds_attn_pruned(pad["q_tail"], pad["k_tail"], pad["v_tail"], pad["k_pre"], pad["v_pre"], idx_t, 0.1,
+                            out=out_big[..., :D])
+    torch.cuda.synchronize()
+    ref = oracle.attn(_np(x["q_tail"]), _np(x["k_tail"]), _np(x["v_tail"]), _np(x["k_pre"]), _np(x["v_pre"]),
+                      np.asarray(idx), 0.1)
+    _compare(out, ref, torch.float32, f"fp32 padded rows D{D}")
+    # a negative scale is inside the fp32 envelope
+    out = ds.ds_attn_pruned(x["q_tail"], x["k_tail"], x["v_tail"], x["k_pre"], x["v_pre"], idx_t, -0.2)
+    ref = oracle.attn(_np(x["q_tail"]), _np(x["k_tail"]), _np(x["v_tail"]), _np(x["k_pre"]), _np(x["v_pre"]),
+                      np.asarray(idx), -0.2)
+    _compare(out, ref, torch.float32, f"fp32 negative scale D{D}")
+
+
+def test_requests_outside_the_envelope_are_refused_not_rerouted():
+    g = torch.Generator().manual_seed(1)
+    mk = lambda D, dt: [torch.randn(1, 2, 64, D, generator=g).to(dt).to(DEV) for _ in range(3)]
+    idx = torch.arange(32, dtype=torch.int32, device=DEV)
+    for D, dt, scale in ((96, torch.bfloat16, 0.1), (32, torch.bfloat16, 0.1), (128, torch.bfloat16, 0.0),
+                         (128, torch.bfloat16, -0.1), (96, torch.float32, 0.1), (160, torch.float32, 0.1)):
+        q, k, v = mk(D, dt)
+        n0 = ds.ds_launch_count()
+        with pytest.raises(ds.DsError) as e:
+            ds.ds_attn_pruned(q, k, v, None, None, idx, scale)
+        assert e.value.code == ds.DS_ERR_UNSUPPORTED and ds.ds_launch_count() == n0, (D, dt, scale)
 
 
 def test_scattered_and_per_batch_index_lists():
@@ -199,9 +281,9 @@ def test_out_of_range_index_sets_status_and_gpu_stays_healthy():
 
 
 # ---------------------------------------------------------------------------
-# full-size configurations, sampled
+# full-size configurations
 # ---------------------------------------------------------------------------
-def _sampled_parity(cfg, n_slices=8, q_rows=None, layer=0, seed=0):
+def _launch_full(cfg, layer=0):
     x = wl.attention_inputs(cfg, device=DEV, layer=layer)
     idx = ds.retained_indices(cfg.gen, cfg.K, 0, cfg.w, cfg.keep_last)
     idx_t = torch.tensor(idx, dtype=torch.int32, device=DEV)
@@ -212,14 +294,32 @@ def _sampled_parity(cfg, n_slices=8, q_rows=None, layer=0, seed=0):
     torch.cuda.synchronize()
     assert ds.ds_read_status(status) == 0
     assert torch.isfinite(out.float()).all()
-    rng = np.random.default_rng(seed)
+    return x, np.asarray(idx), scale, out
+
+
+def _slices_at_cta_boundaries(cfg, n_slices, rng):
+    """(batch, head) pairs to compare: the corners, the heads whose work items are the first and the last of
+    several CTAs' item lists (CTA c of a persistent launch takes items c, c + #SMs, ...; items are numbered
+    batch-major, then KV head), and seeded random ones up to n_slices."""
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    G = cfg.Hq // cfg.Hkv
+    heads_kv = cfg.B * cfg.Hkv
     pairs = {(0, 0), (cfg.B - 1, cfg.Hq - 1), (0, cfg.Hq - 1), (cfg.B - 1, 0)}
+    for item in (0, 1, n_sm - 1, n_sm, n_sm + 1, 2 * n_sm - 1, 2 * n_sm, heads_kv - n_sm, heads_kv - 2, heads_kv - 1):
+        if 0 <= item < heads_kv:
+            b, hk = divmod(item, cfg.Hkv)
+            pairs.add((b, hk * G + int(rng.integers(G))))
     while len(pairs) < min(n_slices, cfg.B * cfg.Hq):
         pairs.add((int(rng.integers(cfg.B)), int(rng.integers(cfg.Hq))))
+    return sorted(pairs)
+
+
+def _sampled_parity(cfg, n_slices=32, q_rows=None, layer=0, seed=0):
+    x, ia, scale, out = _launch_full(cfg, layer)
+    rng = np.random.default_rng(seed)
     G = cfg.Hq // cfg.Hkv
-    ia = np.asarray(idx)
     worst = 0.0
-    for b, h in sorted(pairs):
+    for b, h in _slices_at_cta_boundaries(cfg, n_slices, rng):
         g = h // G
         sl = lambda t, hh: _np(t[b:b + 1, hh:hh + 1])
         q, kt, vt = sl(x["q_tail"], h), sl(x["k_tail"], g), sl(x["v_tail"], g)
@@ -230,10 +330,10 @@ def _sampled_parity(cfg, n_slices=8, q_rows=None, layer=0, seed=0):
         else:
             # sampled query rows: softmax attention does not depend on key order, so the keys of the
             # retained rows that are not sampled are handed to the oracle as extra prefix rows
-            pick = np.sort(rng.choice(len(idx), q_rows, replace=False))
-            pick[0], pick[-1] = 0, len(idx) - 1
+            pick = np.sort(rng.choice(len(ia), q_rows, replace=False))
+            pick[0], pick[-1] = 0, len(ia) - 1
             pick = np.unique(pick)
-            rest = np.setdiff1d(np.arange(len(idx)), pick)
+            rest = np.setdiff1d(np.arange(len(ia)), pick)
             kp2 = np.concatenate([kp, kt[:, :, ia[rest]]], 2)
             vp2 = np.concatenate([vp, vt[:, :, ia[rest]]], 2)
             ref = oracle.attn(q, kt, vt, kp2, vp2, ia[pick], scale)[0, 0]
@@ -243,32 +343,45 @@ def _sampled_parity(cfg, n_slices=8, q_rows=None, layer=0, seed=0):
     return worst
 
 
-@pytest.mark.parametrize("name", ["llada1", "dream16", "long32-w0", "long32-w64", "long32-w256"])
+@pytest.mark.parametrize("name", ["long32-w64", "long32-w0"])
+def test_long_context_bench_workloads_every_slice(name):
+    """The bench workload and its w = 0 companion, in the launch configuration the bench times, compared on
+    all B x Hq = 1024 (batch, head) slices: every persistent CTA's whole item list (7 items of 33 KV tiles
+    through one ring) is covered, not a sample."""
+    cfg = wl.CONFIGS[name]
+    x, ia, scale, out = _launch_full(cfg)
+    for b in range(cfg.B):      # one batch at a time keeps the fp32 host copies small
+        sl = lambda t: _np(t[b:b + 1])
+        ref = oracle.attn(sl(x["q_tail"]), sl(x["k_tail"]), sl(x["v_tail"]), sl(x["k_pre"]), sl(x["v_pre"]), ia, scale)
+        _compare(out[b:b + 1], ref, x["q_tail"].dtype, f"{name} b{b} all heads")
+
+
+@pytest.mark.parametrize("name", ["llada1", "dream16", "long32-w256"])
 def test_full_size_configs_sampled(name):
-    _sampled_parity(wl.CONFIGS[name], n_slices=8)
+    _sampled_parity(wl.CONFIGS[name], n_slices=32)
 
 
 def test_full_size_llada_batched_layers():
     cfg = wl.CONFIGS["llada8x32"]
     for layer in (0, 13, 31):           # independent seeded caches; three of the 32 sampled
-        _sampled_parity(cfg, n_slices=6, layer=layer, seed=layer)
+        _sampled_parity(cfg, n_slices=32, layer=layer, seed=layer)
 
 
 def test_full_size_unpruned_reference_sampled_rows():
     # "all 4032": the window covers the whole suffix; Lq = 4096, Lkv = 8192
-    _sampled_parity(wl.CONFIGS["long32-all"], n_slices=4, q_rows=16)
+    _sampled_parity(wl.CONFIGS["long32-all"], n_slices=32, q_rows=16)
 
 
 def test_cache_refresh_step_dense_no_prefix():
     # first step of a block: no cached prefix, every row of the sequence is a query and a key (Lq = Lkv = 2048)
-    _sampled_parity(wl.CONFIGS["refresh8"], n_slices=4, q_rows=16)
+    _sampled_parity(wl.CONFIGS["refresh8"], n_slices=32, q_rows=16)
 
 
 @pytest.mark.parametrize("path,dtype,Lq", [("simt", torch.float32, 40), ("tc", torch.bfloat16, 97),
                                            ("tc", torch.bfloat16, 300), ("tc2", torch.bfloat16, 300)])
-def test_listed_sequences_only(path, dtype, Lq, monkeypatch):
+def test_listed_sequences_only(path, dtype, Lq):
     # a step restricted to the sequences whose block is unfinished: list and count on the device
-    monkeypatch.setenv("DS_ATTN_PATH", path)
+    kernel = KERNELS.get(path, ds.DS_ATTN_KERNEL_AUTO)     # "simt" = the fp32 kernel, chosen by the element type
     B, Hq, Hkv, D, P, T = 5, 4, 2, 128, 200, 320
     g = torch.Generator().manual_seed(77)
     mk = lambda *sh: torch.randn(*sh, generator=g).to(dtype).to(DEV)
@@ -284,7 +397,7 @@ def test_listed_sequences_only(path, dtype, Lq, monkeypatch):
         status = torch.zeros(1, dtype=torch.int32, device=DEV)
         cnt = None if n_dev is None else torch.tensor([n_dev], dtype=torch.int32, device=DEV)
         ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, out=out, status=status, seq_list=lst, n_seq=n_host,
-                          n_seq_dev=cnt)
+                          n_seq_dev=cnt, kernel=kernel)
         torch.cuda.synchronize()
         assert ds.ds_read_status(status) == 0
         live = lst[: (n_host if n_dev is None else n_dev)].cpu().tolist()
@@ -296,14 +409,14 @@ def test_listed_sequences_only(path, dtype, Lq, monkeypatch):
     # a sequence number outside [0, B) is reported
     bad = torch.tensor([1, 9], dtype=torch.int32, device=DEV)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, status=status, seq_list=bad)
+    ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, status=status, seq_list=bad, kernel=kernel)
     torch.cuda.synchronize()
     assert ds.ds_read_status(status) & ds.DS_DEV_INDEX
 
 
 @pytest.mark.parametrize("path,dtype", [("simt", torch.float32), ("tc", torch.bfloat16), ("tc2", torch.bfloat16)])
-def test_plan_launches_repeat_the_one_shot_call(path, dtype, monkeypatch):
-    monkeypatch.setenv("DS_ATTN_PATH", path)
+def test_plan_launches_repeat_the_one_shot_call(path, dtype):
+    kernel = KERNELS.get(path, ds.DS_ATTN_KERNEL_AUTO)
     B, Hq, Hkv, D, P, T, Lq = 3, 4, 2, 128, 150, 400, 261
     g = torch.Generator().manual_seed(5)
     mk = lambda *sh: torch.randn(*sh, generator=g).to(dtype).to(DEV)
@@ -312,7 +425,7 @@ def test_plan_launches_repeat_the_one_shot_call(path, dtype, monkeypatch):
     scale = 1.0 / math.sqrt(D)
     lst = torch.tensor([0, 2, 1], dtype=torch.int32, device=DEV)
     cnt = torch.tensor([2], dtype=torch.int32, device=DEV)
-    plan = ds.AttnPlan(q, kt, vt, kp, vp, idx, scale, seq_list=lst, n_seq_dev=cnt)
+    plan = ds.AttnPlan(q, kt, vt, kp, vp, idx, scale, seq_list=lst, n_seq_dev=cnt, kernel=kernel)
     n0 = ds.ds_launch_count()
     plan.out.fill_(55.0)
     plan.launch()
@@ -330,16 +443,16 @@ def test_plan_launches_repeat_the_one_shot_call(path, dtype, monkeypatch):
     ref = oracle.attn(_np(q), _np(kt), _np(vt), _np(kp), _np(vp), idx.cpu().numpy(), scale)
     for b in range(B):
         _compare(plan.out[b], ref[b], dtype)
-    one_shot = ds.ds_attn_pruned(q, kt, vt, kp, vp, idx, scale)
+    one_shot = ds.ds_attn_pruned(q, kt, vt, kp, vp, idx, scale, kernel=kernel)
     assert torch.equal(one_shot, plan.out)
     del plan
 
 
 @pytest.mark.parametrize("P,Lq,D", [(1500, 97, 128), (2048, 129, 128), (4096, 65, 128), (1400, 136, 128), (3000, 97, 64)])
-def test_few_work_items_split_over_the_keys(P, Lq, D, monkeypatch):
+def test_few_work_items_split_over_the_keys(P, Lq, D):
     # small batches: the KV tiles of an item are split over several CTAs and merged by a second kernel
     # (needs the workspace; without one the same call runs unsplit)
-    monkeypatch.setenv("DS_ATTN_PATH", "tc")
+    one = dict(kernel=ds.DS_ATTN_KERNEL_ONE_TILE)
     B, Hq, Hkv, T = 2, 4, 2, 1100
     g = torch.Generator().manual_seed(P + Lq)
     mk = lambda *sh: torch.randn(*sh, generator=g).to(torch.bfloat16).to(DEV)
@@ -350,14 +463,14 @@ def test_few_work_items_split_over_the_keys(P, Lq, D, monkeypatch):
     idx_t = torch.tensor(idx, device=DEV)
     scale = 1.0 / math.sqrt(D)
     out = torch.empty((B, Hq, Lq, D), dtype=torch.bfloat16, device=DEV)
-    need = ds.ds_attn_pruned_workspace(q, kt, vt, kp, vp, idx_t, scale, out)
+    need = ds.ds_attn_pruned_workspace(q, kt, vt, kp, vp, idx_t, scale, out, **one)
     assert need > 0, "this shape is meant to be split"
     ref, ref_lse = oracle.attn(_np(q), _np(kt), _np(vt), None if kp is None else _np(kp), None if vp is None else _np(vp),
                                idx, scale, want_lse=True)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     lse = torch.empty((B, Hq, Lq), dtype=torch.float32, device=DEV)
     n0 = ds.ds_launch_count()
-    ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, out=out, lse=lse, status=status)   # the binding allocates the workspace
+    ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, out=out, lse=lse, status=status, **one)   # the binding allocates the workspace
     torch.cuda.synchronize()
     assert ds.ds_launch_count() - n0 == 2 and ds.ds_read_status(status) == 0
     _compare(out, ref, torch.bfloat16, f"split P{P} Lq{Lq}")
@@ -365,14 +478,14 @@ def test_few_work_items_split_over_the_keys(P, Lq, D, monkeypatch):
     # no workspace: one launch, same result up to the second rounding of the partial results
     out2 = torch.empty_like(out)
     n0 = ds.ds_launch_count()
-    ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, out=out2, workspace=torch.empty(256, dtype=torch.uint8, device=DEV))
+    ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, out=out2, workspace=torch.empty(256, dtype=torch.uint8, device=DEV), **one)
     torch.cuda.synchronize()
     assert ds.ds_launch_count() - n0 == 1
     _compare(out2, ref, torch.bfloat16)
     # listed sequences with the count on the device: only those are merged
     out3 = torch.full_like(out, 9.0)
     ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, out=out3, seq_list=torch.tensor([1, 0], dtype=torch.int32, device=DEV),
-                      n_seq_dev=torch.tensor([1], dtype=torch.int32, device=DEV))
+                      n_seq_dev=torch.tensor([1], dtype=torch.int32, device=DEV), **one)
     torch.cuda.synchronize()
     _compare(out3[1], ref[1], torch.bfloat16)
     assert (out3[0] == 9.0).all()

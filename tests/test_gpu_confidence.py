@@ -101,6 +101,13 @@ def test_row_list_and_split_rows():
     _check(z, conf, tok, rows)
     untouched = [r for r in range(cfg.rows) if r not in rows]
     assert (conf[untouched] == -1).all() and (tok[untouched] == -1).all()
+    # a list with no entry touches nothing (no list at all would mean every row)
+    conf.fill_(-2.0)
+    tok.fill_(-2)
+    n0 = ds.ds_launch_count()
+    ds.ds_confidence(z, row_list=torch.empty(0, dtype=torch.int32, device=DEV), conf=conf, tok=tok)
+    torch.cuda.synchronize()
+    assert ds.ds_launch_count() == n0 and (conf == -2).all() and (tok == -2).all()
     # one row, widest split over CTAs
     conf1, tok1 = ds.ds_confidence(z[5:6])
     _check(z[5:6], conf1, tok1)

@@ -4,16 +4,20 @@ Some users of this library cannot allocate device memory at the point where they
 runs inside another framework's memory plan, a plugin whose host forbids allocation after start-up),
 so they cannot provide the workspace ds_confidence asks for.  ds_confidence_static keeps that scratch
 in a fixed array inside the library instead.  It runs the same kernel, so its results must equal those
-of ds_confidence on the same logits: token ids bit for bit, confidences within the tolerance the other
-confidence tests use.  The array is shared by all calls and keeps the last call's contents, so the check
-is made on two calls in a row, the second on different logits.
+of ds_confidence on the same logits, and the CPU oracle's: token ids bit for bit, confidences within the
+tolerance the other confidence tests use.  The array is shared by all calls and keeps the last call's
+contents, so the check is made on two calls in a row, the second on different logits.  The claim that sets
+this entry point apart -- the call allocates nothing -- is checked too: the device's free memory and torch's
+allocator counters are the same before and after it.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run every
 other test.  It passes on its own in a fresh process as well as after the others.
 """
+import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2601_17917_b200 as ds
 
 pytestmark = pytest.mark.gpu
@@ -38,10 +42,22 @@ def test_static_scratch_matches_workspace_entry_point_twice(rows, V, dtype):
         want_conf, want_tok = ds.ds_confidence(z)
         conf.fill_(-1.0)
         tok.fill_(-1)
+        torch.cuda.synchronize()
+        if call == 1:       # the first call on a device looks up the scratch address; from then on nothing moves
+            free0 = torch.cuda.mem_get_info()[0]
+            alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+            n_alloc0 = torch.cuda.memory_stats().get("allocation.all.allocated", 0)
         ds.ds_confidence_static(z, conf, tok)
         torch.cuda.synchronize()
+        if call == 1:
+            assert torch.cuda.mem_get_info()[0] == free0, "device memory in use changed across the call"
+            assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (alloc0, reserved0)
+            assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == n_alloc0
         assert torch.equal(tok, want_tok), f"call {call}: token ids differ"
         assert (conf - want_conf).abs().max().item() <= CONF_TOL, f"call {call}"
+        oc, ot = oracle.confidence(z.float().cpu().numpy())
+        assert (tok.cpu().numpy() == ot).all(), f"call {call}: token ids differ from the oracle's"
+        assert np.abs(conf.cpu().numpy().astype(np.float64) - oc).max() <= CONF_TOL, f"call {call}"
 
 
 def test_static_scratch_with_a_row_list_leaves_other_rows_alone():
@@ -59,6 +75,13 @@ def test_static_scratch_with_a_row_list_leaves_other_rows_alone():
     rest = torch.ones(rows, dtype=torch.bool, device=DEV)
     rest[li] = False
     assert (tok[rest] == -1).all() and (conf[rest] == -1.0).all()
+    # a list with no entry touches nothing (it is not the same as "no list", which means every row)
+    conf.fill_(-2.0)
+    tok.fill_(-2)
+    n0 = ds.ds_launch_count()
+    ds.ds_confidence_static(z, conf, tok, row_list=listed[:0])
+    torch.cuda.synchronize()
+    assert ds.ds_launch_count() == n0 and (tok == -2).all() and (conf == -2.0).all()
 
 
 def test_more_rows_than_the_fixed_scratch_serves_is_refused():
