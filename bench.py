@@ -97,6 +97,48 @@ def job_throughput(world, ms_per_step):
     return world * 1e3 / ms_per_step
 
 
+def replica_command(n, argv, port=None):
+    """The command that starts ``n`` ranks of this script on this node, one per GPU (the launch the multi-GPU
+    contract describes: torch.distributed.run, rendezvous on 127.0.0.1)."""
+    if port is None:
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve()), *argv]
+
+
+def spawn_replicas(n, argv):
+    import subprocess
+    return subprocess.call(replica_command(n, argv))
+
+
+def dry_run(args, cfg):
+    """What a multi-rank run adds to a single-GPU one, without a GPU: the ranks come up, each derives its own
+    seeded batch, the slowest rank's (here: made-up) time becomes the job's time, rank 0 prints the line."""
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo")
+    rcfg = rank_config(cfg, rank)
+    seeds = [None] * world
+    if world > 1:
+        dist.all_gather_object(seeds, rcfg.seed)
+    else:
+        seeds = [rcfg.seed]
+    ms = max_over_ranks(1.0 + rank, world, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "metric": METRIC, "n_gpus": world, "value": job_throughput(world, ms),
+                          "unit": "steps/s", "ms_per_step": ms, "scaling": "weak", "rank_seeds": seeds,
+                          "config": {"workload": cfg.name, "parallelism": f"replicas x{world}"}}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # --------------------------------------------------------------------------
 # clock sampling (read-only NVML)
 # --------------------------------------------------------------------------
@@ -171,16 +213,22 @@ class ClockSampler:
 class Step:
     """Device-resident inputs of one configuration and the three C-ABI calls of a step."""
 
-    def __init__(self, cfg, device, compact_tail=False, stages=("attn", "confidence", "select")):
+    def __init__(self, cfg, device, compact_tail=False, stages=("attn", "confidence", "select"), fused_lmhead=False):
         import torch
         self.stages = tuple(stages)
+        self.fused_lmhead = fused_lmhead
         import paper_2601_17917_b200 as ds
         from paper_2601_17917_b200 import workloads as wl
         self.torch, self.ds, self.cfg, self.device = torch, ds, cfg, device
         idx = ds.retained_indices(cfg.gen, cfg.K, 0, cfg.w, cfg.keep_last)
         self.Lq = len(idx)
         self.layers = []
-        for layer in range(cfg.n_layers):
+        # a configuration whose per-step attention inputs would fit in L2 gets independent seeded copies,
+        # rotated from step to step, so that every timed launch streams from HBM
+        foot = attn_algorithmic_bytes(cfg, self.Lq) * cfg.n_layers
+        self.copies = 1 if foot >= 256e6 else min(16, int(math.ceil(256e6 / foot)))
+        self.tick = 0
+        for layer in range(cfg.n_layers * self.copies):
             x = wl.attention_inputs(cfg, device=device, layer=layer)
             if compact_tail:
                 sel = torch.tensor(idx, device=device)
@@ -191,7 +239,14 @@ class Step:
             idx = list(range(self.Lq))
         self.idx = torch.tensor(idx, dtype=torch.int32, device=device)
         self.scale = 1.0 / math.sqrt(cfg.D)
-        self.logits = wl.logits(cfg, device=device)
+        if fused_lmhead:
+            # the widened path: hidden states in, Eq. 4 out, the [rows x V] logits never stored
+            self.hidden, self.weight = wl.lmhead_inputs(cfg, HIDDEN_SIZE.get(cfg.V, 4096), device=device)
+            self.logits = None
+            self.lm_ws = torch.empty(max(ds.ds_lmhead_confidence_workspace(cfg.rows, cfg.V), 256), dtype=torch.uint8,
+                                     device=device)
+        else:
+            self.logits = wl.logits(cfg, device=device)
         x0, m0 = wl.block_state(cfg, "all")
         self.x0, self.m0 = x0.to(device), m0.to(device)
         self.x_block, self.masked = self.x0.clone(), self.m0.clone()
@@ -216,12 +271,16 @@ class Step:
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
 
     def attn(self, layer=0):
-        x = self.layers[layer]
+        x = self.layers[(self.tick % self.copies) * self.cfg.n_layers + layer]
         self.ds.ds_attn_pruned(x["q_tail"], x["k_tail"], x["v_tail"], x["k_pre"], x["v_pre"], self.idx, self.scale,
                                out=self.out, workspace=self.attn_ws, status=self.status)
 
     def confidence(self):
-        self.ds.ds_confidence(self.logits, conf=self.conf, tok=self.tok, workspace=self.conf_ws)
+        if self.fused_lmhead:
+            self.ds.ds_lmhead_confidence(self.hidden, self.weight, conf=self.conf, tok=self.tok, workspace=self.lm_ws,
+                                         status=self.status)
+        else:
+            self.ds.ds_confidence(self.logits, conf=self.conf, tok=self.tok, workspace=self.conf_ws)
 
     def select(self):
         cfg = self.cfg
@@ -248,6 +307,7 @@ class Step:
             self.select()
         if events:
             events[3].record()
+        self.tick += 1
 
 
 def time_resident(step, steps, warmup, sampler, barrier):
@@ -286,18 +346,63 @@ def time_resident(step, steps, warmup, sampler, barrier):
     return total_ms, stage_ms, launches, windows, extra
 
 
-def time_e2e(cfg, device, steps, warmup, cache_resident=False):
+def time_attn_sustained(step, device_index, seconds=2.0, chunk=64):
+    """The attention stage alone, back to back for at least ``seconds``: long enough for the power cap to settle
+    the SM clock.  CUDA events every ``chunk`` launches; clocks sampled over the same window.  Returns the mean
+    launch time of the whole region and of its second half, with the median SM clock of each."""
+    torch = step.torch
+    for _ in range(3):
+        step.attn(0)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(device_index)
+    sampler.start()
+    evs = [torch.cuda.Event(enable_timing=True)]
+    evs[0].record()
+    t0 = time.perf_counter()
+    stamps = [t0]                            # host time at which chunk i - 1 had finished
+    n = 0
+    while True:
+        for i in range(chunk):
+            step.attn((n + i) % step.cfg.n_layers)
+            if (n + i + 1) % step.cfg.n_layers == 0:
+                step.tick += 1
+        n += chunk
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        evs.append(e)
+        evs[-2].synchronize()                # the chunk before this one is done; this one keeps the GPU busy
+        stamps.append(time.perf_counter())
+        if stamps[-1] - t0 >= seconds:
+            break
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    sampler.stop()
+    k = len(evs) - 1
+    whole_ms = evs[0].elapsed_time(evs[k])
+    half = k // 2
+    tail_ms = evs[half].elapsed_time(evs[k])
+    cl_all = sampler.summary([(t0, t1)])
+    cl_tail = sampler.summary([(stamps[half], t1)])
+    return {"launches": n, "seconds": whole_ms * 1e-3, "us_per_launch": whole_ms * 1e3 / n,
+            "sm_mhz": cl_all["sm_mhz"], "reasons": cl_all["reasons"],
+            "second_half": {"launches": n - half * chunk, "us_per_launch": tail_ms * 1e3 / max(1, n - half * chunk),
+                            "sm_mhz": cl_tail["sm_mhz"]}}
+
+
+def time_e2e(cfg, device, steps, warmup, cache_resident=False, fused_lmhead=False):
     """Same step from pinned host buffers: H2D of everything the step reads, the three calls,
     D2H of the results, all inside the timed region.  ``cache_resident``: the prefix KV cache stays on
     the device (the method computes it once per block and reuses it at every step); only what changes
-    from step to step is copied."""
+    from step to step is copied.  ``fused_lmhead``: the step ends in ds_lmhead_confidence instead of
+    ds_confidence, so the hidden states of the block's rows cross the link instead of their logits (the output
+    embedding stays on the device like any weight)."""
     import torch
-    dev_step = Step(cfg, device, compact_tail=True)
+    dev_step = Step(cfg, device, compact_tail=True, fused_lmhead=fused_lmhead)
     host_in, dev_in = [], []
     for x in dev_step.layers:
         for k in ("q_tail", "k_tail", "v_tail") + (() if cache_resident else ("k_pre", "v_pre")):
             dev_in.append(x[k])
-    dev_in += [dev_step.logits, dev_step.x_block, dev_step.masked, dev_step.idx]
+    dev_in += [dev_step.hidden if fused_lmhead else dev_step.logits, dev_step.x_block, dev_step.masked, dev_step.idx]
     for t in dev_in:
         h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
         h.copy_(t)
@@ -564,6 +669,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the extra timing of ds_lmhead_confidence")
     ap.add_argument("--no-decode-loop", action="store_true", help="skip the extra timing of the block-wise decode loop")
+    ap.add_argument("--no-sustained", action="store_true",
+                    help="skip the seconds-long attention-only region behind `roofline_sustained`")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0)
+    ap.add_argument("--dry-run", action="store_true",
+                    help="launch plumbing only: ranks, seeds and the max-over-ranks reduction on CPU (gloo), no GPU work")
     ap.add_argument("--stages", default="attn,confidence,select",
                     help="comma list of the stages a step runs (profiling a single kernel)")
     ap.add_argument("--vocab", type=int, default=0, help="override the vocabulary size (small profiler cases)")
@@ -579,6 +689,12 @@ def main():
         cfg = wl.shrink(cfg, V=args.vocab, name=f"{cfg.name}-V{args.vocab}")
     if args.impl == "reference":
         run_reference(args, cfg)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started bare: become the launcher of N ranks (one per GPU) and pass their exit code on
+        raise SystemExit(spawn_replicas(args.gpus, sys.argv[1:]))
+    if args.dry_run:
+        dry_run(args, cfg)
         return
 
     import torch
@@ -622,6 +738,10 @@ def main():
     clocks = sampler.summary(windows)
     if extra:
         clocks["note"] = f"timed region + {extra} further identical steps"
+    sustained = None
+    if not args.no_sustained and "attn" in step.stages and args.sustained_seconds > 0:
+        sustained = time_attn_sustained(step, local, seconds=args.sustained_seconds)
+        barrier()
     status = ds.ds_read_status(step.status)
     total_ms = max_over_ranks(total_ms, world, device)
     ms_per_step = total_ms / args.steps
@@ -630,7 +750,7 @@ def main():
     e2e = None
     if not args.no_e2e and args.stages == "attn,confidence,select":
         e2e_steps = max(3, min(args.steps, 20))
-        del step.layers[1:]
+        step.layers.clear()
         torch.cuda.empty_cache()
         e_ms, h2d, d2h = time_e2e(rcfg, device, e2e_steps, 3)
         e_ms = max_over_ranks(e_ms, world, device)
@@ -642,6 +762,14 @@ def main():
         r_ms = max_over_ranks(r_ms, world, device)
         e2e["prefix_cache_resident"] = {"value": job_throughput(world, r_ms), "unit": "steps/s", "ms_per_step": r_ms,
                                         "h2d_bytes_per_step": int(r_h2d), "d2h_bytes_per_step": int(r_d2h)}
+        # third figure: cache resident and the step ending in the fused output projection (hidden states in)
+        if cfg.dtype == "bf16":
+            f_ms, f_h2d, f_d2h = time_e2e(rcfg, device, e2e_steps, 3, cache_resident=True, fused_lmhead=True)
+            f_ms = max_over_ranks(f_ms, world, device)
+            e2e["fused_lmhead"] = {"value": job_throughput(world, f_ms), "unit": "steps/s", "ms_per_step": f_ms,
+                                   "h2d_bytes_per_step": int(f_h2d), "d2h_bytes_per_step": int(f_d2h),
+                                   "what": "prefix cache and output embedding resident; hidden states of the block's rows "
+                                           "copied in; ds_lmhead_confidence in place of logits + ds_confidence"}
 
     if rank != 0:
         if world > 1:
@@ -689,6 +817,24 @@ def main():
                                 "algorithmic_bytes": c_bytes},
         "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
     }
+    if clocks.get("sm_mhz"):
+        line["roofline"]["us_per_launch"] = a_ms * 1e3
+        line["roofline"]["us_x_mhz"] = a_ms * 1e3 * clocks["sm_mhz"]
+    if sustained is not None:
+        # the same kernel over seconds of back-to-back launches: the power cap has settled the SM clock, so this is
+        # the figure a long-running decode sees; time x clock says how much of the difference is the clock
+        def entry(us, mhz):
+            if attn_roof["bound"] == "hbm":
+                ach, peak, unit = a_bytes / (us * 1e-6) / 1e9, pk["hbm_gbs"], "GB/s"
+            else:
+                ach, peak, unit = fl / (us * 1e-6) / 1e12, pk["bf16_tflops_sustained"], "TFLOP/s"
+            return {"achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "us_per_launch": us, "sm_mhz": mhz,
+                    "us_x_mhz": us * mhz if mhz else None}
+        rs = entry(sustained["us_per_launch"], sustained["sm_mhz"])
+        rs.update({"kernel": "ds_attn_pruned", "bound": attn_roof["bound"], "seconds": sustained["seconds"],
+                   "launches": sustained["launches"], "reasons": sustained["reasons"], "peak_source": attn_roof["peak_source"],
+                   "second_half": entry(sustained["second_half"]["us_per_launch"], sustained["second_half"]["sm_mhz"])})
+        line["roofline_sustained"] = rs
     if args.stages != "attn,confidence,select":
         line["stages"] = args.stages          # partial step: a profiling run, not a bench value
     if e2e:

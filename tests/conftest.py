@@ -26,5 +26,7 @@ def pytest_terminal_summary(terminalreporter):
         return
     rows = sorted(rows, reverse=True)
     terminalreporter.write_line(f"attention parity: {len(rows)} comparisons, worst max-abs-err / RMS(O):")
-    for ratio, err, rms, what in rows[:8]:
-        terminalreporter.write_line(f"  {ratio:.3e}  (err {err:.3e}, rms {rms:.3e})  {what}")
+    for ratio, err, rms, row_ratio, what in rows[:8]:
+        terminalreporter.write_line(f"  {ratio:.3e}  (err {err:.3e}, rms {rms:.3e}, per-row excess {row_ratio:.3e})  {what}")
+    worst_row = max(r[3] for r in rows)
+    terminalreporter.write_line(f"  worst (|err| - 2^-8 |ref|) / rms of the row, over all comparisons: {worst_row:.3e}")

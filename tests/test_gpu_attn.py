@@ -26,15 +26,20 @@ DEV = "cuda:0"
 ABS_BAR = 1e-2
 
 
-# max-abs-err / RMS(O) of every comparison made in this module: (ratio, err, rms, what)
+# max-abs-err / RMS(O) of every comparison made in this module: (ratio, err, rms, worst row ratio, what)
 ERR_OVER_RMS = []
-# The kernel's own error model, elementwise: |out - ref| <= REL * |ref| + RMS_FRAC * RMS(ref) + ABS.
-#   bf16: REL = 2^-8 (output rounding is 2^-9; the split path rounds partial results once more),
-#         RMS_FRAC = 2.5e-2 (bf16 probabilities: 2^-9 relative each, a few sigma over ~1e6 elements,
-#         plus the approximate exponential), ABS = 1e-6
-#   fp32: REL = 1e-5, RMS_FRAC = 1e-4, ABS = 1e-6
+# The kernel's own error model, elementwise:  |out - ref| <= REL * |ref| + ROW_FRAC * rms_row + ABS,
+# rms_row = RMS over the head dimension of the reference row the element belongs to.
+#   bf16: REL = 2^-8 (output rounding is 2^-9; the split path rounds partial results once more).
+#         ROW_FRAC: the probabilities are rounded to bf16 (2^-9 relative, independent), which perturbs
+#         o_i = sum_j p_ij v_j by about 2^-9 sqrt(sum_j p_ij^2 v_j^2) ~ 2^-9 rms_row_i for unit-variance values
+#         (rms_row_i ~ sqrt(sum_j p_ij^2): it grows with how peaked the row's softmax is, which is why the bound
+#         is per row and not per tensor); the maximum over ~1e6 elements sits 4-5 sigma out, and the
+#         approximate exponential and the lazy rescale add to it.  Measured worst over all cases of this file:
+#         1.3e-2; the bound is twice that, 2.5e-2.  ABS = 1e-6.
+#   fp32: REL = 1e-5, ROW_FRAC = 2e-4, ABS = 1e-6
 def _tol(dtype):
-    return (1e-5, 1e-4, 1e-6) if dtype == torch.float32 else (2.0 ** -8, 2.5e-2, 1e-6)
+    return (1e-5, 2e-4, 1e-6) if dtype == torch.float32 else (2.0 ** -8, 2.5e-2, 1e-6)
 
 
 def _np(t):
@@ -46,12 +51,14 @@ def _compare(out, ref, dtype, what=""):
     diff = np.abs(out - ref)
     err = diff.max()
     rms = math.sqrt(float((ref ** 2).mean())) + 1e-30
-    rel, rms_frac, floor = _tol(dtype)
+    rel, row_frac, floor = _tol(dtype)
     assert np.isfinite(out).all(), what
     # the stated bar: 1e-2 max-abs on unit-scale values (bf16 cannot hold 1e-2 absolute beyond |x| = 2.56)
     assert (diff <= ABS_BAR * np.maximum(1.0, np.abs(ref))).all(), (what, err)
-    ERR_OVER_RMS.append((err / rms, err, rms, what))
-    assert (diff <= rel * np.abs(ref) + rms_frac * rms + floor).all(), (what, err, rms, err / rms)
+    rms_row = np.sqrt((ref ** 2).mean(axis=-1, keepdims=True)) + 1e-30
+    row_ratio = float((np.maximum(diff - rel * np.abs(ref), 0.0) / rms_row).max())
+    ERR_OVER_RMS.append((err / rms, err, rms, row_ratio, what))
+    assert (diff <= rel * np.abs(ref) + row_frac * rms_row + floor).all(), (what, err, rms, row_ratio)
     return err, rms
 
 

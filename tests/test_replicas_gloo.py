@@ -64,3 +64,22 @@ def test_reference_arm_runs_on_rank_0_only():
     line = json.loads(p.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_bare_gpus_flag_starts_its_own_ranks():
+    """`python bench.py --gpus 2` without a launcher around it starts two ranks itself; with --dry-run the ranks
+    do the host-side part only (gloo): own seeds per rank, max over ranks, n_gpus = 2 in the one line printed."""
+    import bench
+    cmd = bench.replica_command(2, ["--gpus", "2", "--dry-run"], port=29431)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-3:] == ["--gpus", "2", "--dry-run"]
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--gpus", "2", "--dry-run", "--config", "tiny"], env=env,
+                       capture_output=True, text=True, timeout=600)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [json.loads(l) for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    line = lines[0]
+    assert line["dry_run"] and line["n_gpus"] == 2 and line["config"]["parallelism"] == "replicas x2"
+    assert len(set(line["rank_seeds"])) == 2                 # every replica draws its own batch
+    assert line["ms_per_step"] == 2.0 and line["value"] == 2 * 1e3 / 2.0     # slowest rank's time; whole-job steps/s
