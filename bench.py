@@ -525,53 +525,91 @@ def time_lmhead(cfg, device, reps=10):
 
 def time_decode_loop(device, n_blocks=8, batches=(8, 1)):
     """The whole block-wise procedure on the LLaDA-shaped configuration (32 layers, prompt 1024, n_blocks blocks
-    of 32; 8 sequences, and 1 as in the paper's per-sample latency figures): per block one refresh iteration
-    (dense attention over prefix + retained rows, every layer) and pruned iterations until the block has no mask
-    left, driven by decode.BlockDecoder.  The model's other layers are absent: the logits of an iteration are
-    staged from a small pool of seeded buffers.  Three ways to drive the same device work: the synchronous loop
-    (the host waits for every iteration), the host running two iterations ahead, and the latter with every
-    iteration replayed as one CUDA graph."""
+    of 32; 8 sequences, and 1 as in the paper's per-sample latency figures), driven by decode.BlockDecoder with
+    the attention side of every layer done as the method does it.  Per layer the seeded buffers are un-rotated
+    Q/K/V projections of every position and a prefix KV cache that starts with the prompt's rows:
+      first iteration of block n   the finished block n-1 joins the cache (ds_rope_gather, n_append = K); dense
+                                   attention over prefix + retained rows with nothing cached (rotary encoding +
+                                   gather of all rows, then ds_attn_pruned with P = 0)
+      later iterations             rotary encoding + gather of the retained tail rows, ds_attn_pruned over the
+                                   cache rows 0 .. P + n K and the retained rows
+    so block n + 1 attends over what block n appended.  The model's other layers are absent: the logits of an
+    iteration are staged from a small pool of seeded buffers.  Three ways to drive the same device work: the
+    synchronous loop (the host waits for every iteration), the host running two iterations ahead, and the latter
+    with every iteration replayed as one CUDA graph."""
     import torch
     import paper_2601_17917_b200 as ds
     from paper_2601_17917_b200 import workloads as wl
     from paper_2601_17917_b200.decode import BlockDecoder
     base = wl.CONFIGS["llada8x32"]
-    res = {"what": "whole block-wise decode (refresh + pruned iterations per block, early exit off); not part of `value`",
+    res = {"what": "whole block-wise decode (per layer: rotary encoding + gather, pruned attention over the growing "
+                   "prefix cache, cache append at every block boundary; early exit off); not part of `value`",
            "blocks": n_blocks, "K": base.K, "n_layers": base.n_layers, "P": base.P, "batches": {}}
     status = torch.zeros(1, dtype=torch.int32, device=device)
+    theta = 10000.0
     for nb in batches:
         cfg = wl.shrink(base, B=nb, gen=n_blocks * base.K, name=f"llada{nb}x32-decode")
-        B, K, L, P, D = cfg.B, cfg.K, cfg.gen, cfg.P, cfg.D
-        layers = [wl.attention_inputs(cfg, device=device, layer=l) for l in range(cfg.n_layers)]
+        B, K, L, P, D, Hq, Hkv = cfg.B, cfg.K, cfg.gen, cfg.P, cfg.D, cfg.Hq, cfg.Hkv
+        dt = cfg.torch_dtype()
+        # per layer: raw projections of prompt + generation, and the cache (prompt rows filled below)
+        raws, caches = [], []
+        for l in range(cfg.n_layers):
+            x = wl.attention_inputs(wl.shrink(cfg, P=0, gen=P + L, name="raw"), device=device, layer=l)
+            raws.append((x["q_tail"], x["k_tail"], x["v_tail"]))
+            caches.append((torch.zeros((B, Hkv, P + L, D), dtype=dt, device=device),
+                           torch.zeros((B, Hkv, P + L, D), dtype=dt, device=device)))
         pool = [wl.logits(cfg, device=device, step=s, spike_range=(14.0, 26.0)) for s in range(4)]
         scale = 1.0 / math.sqrt(D)
         Lq_max = len(ds.retained_indices(L, K, 0, cfg.w, cfg.keep_last))
-        # refresh iteration: queries and keys are all of prefix + retained rows (one seeded set shared by the layers)
-        dense = wl.attention_inputs(wl.shrink(cfg, P=0, gen=P + Lq_max, name="refresh"), device=device, layer=99)
-        out = torch.empty((B, cfg.Hq, P + Lq_max, D), dtype=cfg.torch_dtype(), device=device)
-        ar = torch.arange(P + Lq_max, dtype=torch.int32, device=device)
+        n_max = P + L                                    # rows of a refresh iteration never exceed the sequence
+        # compact rotated rows of the layer being processed (shared by the layers: they run one after another)
+        qc = torch.empty((B, Hq, n_max, D), dtype=dt, device=device)
+        kc = torch.empty((B, Hkv, n_max, D), dtype=dt, device=device)
+        vc = torch.empty((B, Hkv, n_max, D), dtype=dt, device=device)
+        out = torch.empty((B, Hq, n_max, D), dtype=dt, device=device)
+        ar = torch.arange(n_max, dtype=torch.int32, device=device)
+        rows_all = {}                                    # block -> rows of its refresh iteration (absolute positions)
+        for n in range(n_blocks):
+            keep = torch.tensor(ds.retained_indices(L, K, n, cfg.w, cfg.keep_last), dtype=torch.int32, device=device)
+            rows_all[n] = torch.cat([ar[:P + n * K], keep + (P + n * K)])
+
+        def prefill():
+            for (q, k, v), (ck, cv) in zip(raws, caches):
+                ds.ds_rope_gather(q, k, v, ar[:P], 0, theta, q_out=qc[:, :, :P], k_out=kc[:, :, :P], v_out=vc[:, :, :P],
+                                  k_cache=ck, v_cache=cv, cache_row0=0, n_append=P, status=status)
 
         def forward_for(dec):
-            # the calls of a block repeat with the same pointers: plan them once per block
+            # the attention calls of a block repeat with the same pointers: plan them once per block
             plans = {}
 
             def forward(st):
-                key = (st.n, st.refresh)
-                if key not in plans:
-                    if st.refresh:
-                        n_rows = P + len(ds.retained_indices(L, K, st.n, cfg.w, cfg.keep_last))
-                        one = ds.AttnPlan(dense["q_tail"], dense["k_tail"], dense["v_tail"], None, None, ar[:n_rows],
-                                          scale, out=out[:, :, :n_rows], status=status, seq_list=st.active_seq, n_seq=B,
-                                          n_seq_dev=st.active_cnt)
-                        plans[key] = [one] * cfg.n_layers
-                    else:
-                        r0 = st.n * K
-                        plans[key] = [ds.AttnPlan(x["q_tail"][:, :, r0:], x["k_tail"][:, :, r0:], x["v_tail"][:, :, r0:],
-                                                  x["k_pre"], x["v_pre"], st.idx, scale, out=out[:, :, :st.idx.numel()],
-                                                  status=status, seq_list=st.active_seq, n_seq=B,
-                                                  n_seq_dev=st.active_cnt) for x in layers]
-                for pl in plans[key]:
-                    pl.launch()
+                n, b0 = st.n, P + st.n * K               # b0: rows of the cache in use = position of tail row 0
+                key = (n, st.refresh)
+                if st.refresh:
+                    rows = rows_all[n]
+                    nr = rows.numel()
+                    if key not in plans:
+                        plans[key] = ds.AttnPlan(qc[:, :, :nr], kc[:, :, :nr], vc[:, :, :nr], None, None, ar[:nr], scale,
+                                                 out=out[:, :, :nr], status=status, seq_list=st.active_seq, n_seq=B,
+                                                 n_seq_dev=st.active_cnt)
+                    for (q, k, v), (ck, cv) in zip(raws, caches):
+                        if n > 0:                        # the finished block joins the prefix
+                            ds.ds_rope_gather(q[:, :, b0 - K:], k[:, :, b0 - K:], v[:, :, b0 - K:], ar[:K], b0 - K, theta,
+                                              q_out=qc[:, :, :K], k_out=kc[:, :, :K], v_out=vc[:, :, :K], k_cache=ck,
+                                              v_cache=cv, cache_row0=b0 - K, n_append=K, status=status)
+                        ds.ds_rope_gather(q, k, v, rows, 0, theta, q_out=qc[:, :, :nr], k_out=kc[:, :, :nr],
+                                          v_out=vc[:, :, :nr], status=status)
+                        plans[key].launch()
+                else:
+                    lq = st.idx.numel()
+                    if key not in plans:
+                        plans[key] = [ds.AttnPlan(qc[:, :, :lq], kc[:, :, :lq], vc[:, :, :lq], ck[:, :, :b0], cv[:, :, :b0],
+                                                  ar[:lq], scale, out=out[:, :, :lq], status=status, seq_list=st.active_seq,
+                                                  n_seq=B, n_seq_dev=st.active_cnt) for ck, cv in caches]
+                    for (q, k, v), pl in zip(raws, plans[key]):
+                        ds.ds_rope_gather(q[:, :, b0:], k[:, :, b0:], v[:, :, b0:], st.idx, b0, theta, q_out=qc[:, :, :lq],
+                                          k_out=kc[:, :, :lq], v_out=vc[:, :, :lq], status=status)
+                        pl.launch()
             return forward
 
         runs = {}
@@ -580,6 +618,7 @@ def time_decode_loop(device, n_blocks=8, batches=(8, 1)):
                                keep_last=cfg.keep_last, device=device, lookahead=la)
             forward = forward_for(dec)
             stage = lambda n, t: dec.logits.copy_(pool[(n + t) % len(pool)])
+            prefill()
             dec.decode(forward, before_iteration=stage, graphs=graphs)      # warm-up: plans, graph capture
             torch.cuda.synchronize()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -595,7 +634,7 @@ def time_decode_loop(device, n_blocks=8, batches=(8, 1)):
                           "host_launch_calls": int(ds.ds_launch_count() - n0)}
             del dec, forward
         res["batches"][f"B{nb}"] = runs
-        del layers, pool, dense, out
+        del raws, caches, pool, qc, kc, vc, out
         torch.cuda.empty_cache()
     res["device_status"] = int(ds.ds_read_status(status))
     return res

@@ -16,12 +16,12 @@
 // reduction per tile; instead those columns are expressed against a reference exponent that is only
 // moved (with an exact rescale) when a score exceeds it by more than 2^24.
 //
-// Warp roles (480 threads, one CTA per SM):
+// Warp roles (512 threads, one CTA per SM):
 //   warps 0-7  softmax + epilogue.  Warp w works on the 16 TMEM lanes 32 (w % 4) + 16 (w / 4) ..;
 //              two threads share a row (lanes l and l + 16 of the warp take the two column halves of
 //              every S tile, tcgen05.ld shape 16x32bx2), so a row maximum is one shuffle away and
 //              every scheduler has two softmax warps.
-//   warp  8    TMA producer (lane 0 issues; the warp stages the index list of each gathered tile)
+//   warp  8    TMA producer of the K/V tiles (lane 0 issues; the warp stages the index list of each gathered tile)
 //   warp  9    TMEM allocation; issues Q K^T (one elected lane)
 //   warps 10-13 softmax + epilogue of the transposed problem (thread = key of the tile; idle in items
 //              without extra rows), kept apart so that its cross-warp agreement never sits on the
@@ -29,6 +29,11 @@
 //   warp 14    issues P V.  Issuing blocks while the tensor pipe's queue is full, so the two streams
 //              have an issuer each; the one dependency the pipe no longer orders by itself (Q K^T of
 //              tile g + 2 overwrites the buffer P V of tile g reads) is an explicit barrier wait.
+//   warp 15    TMA producer of the query tiles.  Gathering a query tile takes the issuing warp about as long
+//              as a KV tile lasts, so it has a warp of its own: the K/V stream starts at once and never
+//              pauses for it.  In the kQ2 instantiation (items of few KV tiles) there are two query buffers
+//              and four ring slots instead of one and five: the next item's queries are then fetched while
+//              the current item runs, which removes the stall at every item boundary.
 // Per KV tile:  S[g%2] = Q K^T            (tcgen05.mma, both operands K-major in shared memory)
 //               softmax warps: tcgen05.ld S, row maximum, P = 2^(s*c - m) as bf16 written over the
 //               first 64 columns of the same S buffer
@@ -64,28 +69,33 @@ using namespace attn;
 
 constexpr int kSoftmaxWarps = 8;
 constexpr int kXWarps = 4;  // softmax of the transposed problem (one per TMEM lane quadrant)
-constexpr int kNumThreads = (kSoftmaxWarps + 3 + kXWarps) * 32;
+constexpr int kNumThreads = (kSoftmaxWarps + 4 + kXWarps) * 32;
 constexpr int kProducerWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1, kXWarp0 = kSoftmaxWarps + 2;
 constexpr int kPvWarp = kXWarp0 + kXWarps;  // second MMA issuer
+constexpr int kQWarp = kPvWarp + 1;         // producer of the query tiles
 constexpr int kXRows = 16;                  // N of the transposed problem (the smallest N for M = 128)
 constexpr int kXMax = 8;                    // extra rows actually served
 constexpr int kXChunkBytes = kXRows * 128;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
+constexpr int kQ2MaxTiles = 24;             // items of at most this many KV tiles get the two-query-buffer instantiation
 constexpr float kXLimit = 24.0f;            // log2 units a transposed score may exceed its reference by
 
-template <int D>
+template <int D, bool kQ2>
 struct Geo {
   static constexpr int kChunks = D / 64;                    // 64-column chunks per tile
   static constexpr int kTileBytes = kChunks * kChunkBytes;  // Q / K / V tile
-  static constexpr int kSlots = (D == 128) ? 5 : 10;        // ring of K/V tiles
-  static constexpr int kOffQ = 0;
-  static constexpr int kOffQx = kTileBytes;                 // [kChunks][16 rows][128 B]
-  static constexpr int kOffPx = kOffQx + 2 * kXChunkBytes;  // [2 buffers][2 chunks][16 rows][128 B]
+  static constexpr int kQBufs = kQ2 ? 2 : 1;                // query buffers (by item parity)
+  static constexpr int kSlots = ((D == 128) ? 5 : 10) - (kQ2 ? (D == 128 ? 1 : 2) : 0);  // ring of K/V tiles
+  static constexpr int kOffQ = 0;                           // [kQBufs] tiles
+  static constexpr int kQxBytes = 2 * kXChunkBytes;         // small query tile: [2 chunks][16 rows][128 B]
+  static constexpr int kOffQx = kQBufs * kTileBytes;        // [kQBufs] small tiles
+  static constexpr int kOffPx = kOffQx + kQBufs * kQxBytes;  // [2 buffers][2 chunks][16 rows][128 B]
   static constexpr int kOffRing = kOffPx + 4 * kXChunkBytes;
   static constexpr int kOffBar = kOffRing + kSlots * kTileBytes;
   // barriers: q_full, q_free, s_full[2], p_full[2], pv_done[2], o_free, xbar[2], ybar, o_full, px_full[2],
-  //           ox_free, sx_full[2], pvx_done[2], slot_full[kSlots], slot_empty[kSlots]
-  static constexpr int kNumBars = 20 + 2 * kSlots;
+  //           ox_free, sx_full[2], pvx_done[2], slot_full[kSlots], slot_empty[kSlots], q_full / q_free of the
+  //           second query buffer
+  static constexpr int kNumBars = 22 + 2 * kSlots;
   static constexpr int kOffIdx = kOffBar + 8 * kNumBars;     // int32[128] gathered-row indices of a KV tile
   static constexpr int kOffIdxQ = kOffIdx + 4 * 128;         // int32[128] gathered-row indices of a query tile
   static constexpr int kOffXflag = kOffIdxQ + 4 * 128;       // int[2 parity][4 warps]
@@ -97,13 +107,14 @@ struct Geo {
   static constexpr int kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;  // P(g) overwrites columns 0..63 of S(g)
   static constexpr int kTmemSx0 = 384, kTmemSx1 = 400, kTmemOx = 416;
 };
-static_assert(Geo<128>::kSmemBytes <= 227 * 1024, "shared memory budget");
-static_assert(Geo<64>::kSmemBytes <= 227 * 1024, "shared memory budget");
+static_assert(Geo<128, false>::kSmemBytes <= 227 * 1024 && Geo<128, true>::kSmemBytes <= 227 * 1024, "shared memory budget");
+static_assert(Geo<64, false>::kSmemBytes <= 227 * 1024 && Geo<64, true>::kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct TcParams : attn::AttnCommon {
   int n_mtiles;  // M-tiles per (batch, KV head)
   int x_rows;    // extra rows riding with the last M-tile (0 = none)
   int n_items;   // B * Hkv * n_mtiles * splits
+  int q2;        // 1: several items per CTA and few KV tiles per item: the instantiation with two query buffers
   // Few work items (small batches): the KV tiles of an item are split over `splits` CTAs, each writing a
   // normalised partial result and its log-sum-exp to the workspace (out / lse then point there, one copy per
   // split, split_stride elements apart); a second kernel merges them.
@@ -142,9 +153,9 @@ __device__ __forceinline__ Item decode_item(const TcParams &prm, int item) {
 // ------------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------------
-template <int D, bool kSplit>
+template <int D, bool kSplit, bool kQ2>
 __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_constant__ TcParams prm) {
-  using G_ = Geo<D>;
+  using G_ = Geo<D, kQ2>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -166,6 +177,12 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
   const uint32_t bar_pvx_done = bar0 + 144;  // [2] O_x^T += V^T P_x^T of a tile has completed
   const uint32_t bar_slot_full = bar0 + 160;                       // [kSlots]
   const uint32_t bar_slot_empty = bar_slot_full + 8 * G_::kSlots;  // [kSlots]
+  const uint32_t bar_q1 = bar_slot_empty + 8 * G_::kSlots;         // q_full, q_free of the second query buffer
+  // query buffer of this CTA's k-th item, its two barriers and their phase for that item
+  auto q_buf = [](int k) { return kQ2 ? (k & 1) : 0; };
+  auto q_phase = [](int k) { return (uint32_t)(kQ2 ? (k >> 1) & 1 : k & 1); };
+  auto q_full_bar = [&](int k) { return q_buf(k) ? bar_q1 : bar_q_full; };
+  auto q_free_bar = [&](int k) { return q_buf(k) ? bar_q1 + 8 : bar_q_free; };
   int32_t *idx_s = reinterpret_cast<int32_t *>(smem + G_::kOffIdx);
   int32_t *idxq_s = reinterpret_cast<int32_t *>(smem + G_::kOffIdxQ);
   volatile uint32_t *tmem_base_s = reinterpret_cast<volatile uint32_t *>(smem + G_::kOffMisc);
@@ -178,6 +195,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
   if (tid == 0) {
     mbar_init(bar_q_full, 1);
     mbar_init(bar_q_free, 1);
+    mbar_init(bar_q1, 1);
+    mbar_init(bar_q1 + 8, 1);
     mbar_init(bar_s_full, 1);
     mbar_init(bar_s_full + 8, 1);
     mbar_init(bar_p_full, kSoftmaxWarps);
@@ -214,7 +233,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
   bool timed_out = false;
 
   if (warp == kProducerWarp) {
-    // ============================ TMA producer ============================
+    // ============================ TMA producer: K/V tiles ============================
     bool bad_index = attn::bad_sequence_numbers(prm, n_live);
     if (lane == 0) {
       auto prefetch_map = [](const CUtensorMap *m) {
@@ -228,39 +247,15 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       prefetch_map(&prm.k1);
       prefetch_map(&prm.v32);
       prefetch_map(&prm.v1);
-      prefetch_map(&prm.q32);
-      prefetch_map(&prm.q1);
       prefetch_map(&prm.k128);
       prefetch_map(&prm.v128);
-      prefetch_map(&prm.q128);
     }
-    // one index list for all batches: keep (the head of) it in shared memory, validated once
+    // One index list for all batches: (the head of) it is kept in shared memory, validated once -- but only
+    // when the first tail tile comes up, so that the prefix tiles are requested without waiting for it.
     const int32_t *idx_cache = nullptr;
     bool list_ok = false;  // the list is known to be in range and strictly ascending
-    if (prm.idx_bstride == 0) {
-      int32_t *cache = reinterpret_cast<int32_t *>(smem + G_::kOffIdxCache);
-      list_ok = cache_shared_index_list(prm, cache, bad_index);
-      __syncwarp();
-      if (list_ok) idx_cache = cache;  // a malformed list is read entry by entry from global memory
-    }
+    bool list_seen = false;
     const int n_my = (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // items of this CTA
-    int q_next = 0;  // first item (in this CTA's order) whose query tile has not been requested yet
-    // Requests the query tile(s) of this CTA's kq-th item.  The caller has made sure the previous
-    // item's last Q K^T has completed.
-    auto issue_q = [&](int kq) {
-      const Item it = decode_item<kSplit>(prm, blockIdx.x + kq * gridDim.x);
-      uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
-                                      it.mt * kBlockM, it.m_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index);
-      if (it.x_rows > 0) {
-        // rows of the small query tile that are not loaded must be finite: clear the tile first
-        for (int q = lane; q < (2 * kXChunkBytes) / 16; q += 32)
-          *reinterpret_cast<uint4 *>(smem + G_::kOffQx + q * 16) = make_uint4(0, 0, 0, 0);
-        fence_proxy_async();
-        bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQx, kXChunkBytes, bar_q_full,
-                                (it.mt + 1) * kBlockM, it.x_rows, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index);
-      }
-      if (lane == 0) mbar_arrive_expect_tx(bar_q_full, bytes);
-    };
     int issued = 0;  // ring fills issued so far
     for (int k = 0; k < n_my && !timed_out; ++k) {
       const Item it = decode_item<kSplit>(prm, blockIdx.x + k * gridDim.x);
@@ -271,44 +266,23 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
           const int slot = issued % G_::kSlots, use = issued / G_::kSlots;
           const uint32_t dst = sbase + G_::kOffRing + slot * G_::kTileBytes;
           const uint32_t full = bar_slot_full + 8 * slot;
-          // Wait for the ring slot.  The KV stream runs ahead of the query tiles across item
-          // boundaries, so while waiting, serve the query tile of the item these fills belong to as
-          // soon as the previous item has released the buffer.
-          bool got = false;
-          for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-            if (q_next <= k) {
-              bool ready = (q_next == 0) || mbar_try_wait(bar_q_free, (q_next - 1) & 1);
-              ready = __all_sync(0xffffffffu, ready);
-              if (ready) {
-                issue_q(q_next);
-                ++q_next;
-                continue;
-              }
-            }
-            bool e = mbar_try_wait(bar_slot_empty + 8 * slot, (use & 1) ^ 1);
-            e = __all_sync(0xffffffffu, e);
-            if (e) {
-              got = true;
-              break;
-            }
-            if (spin > 128) {
-              __nanosleep(64);
-              if (__any_sync(0xffffffffu, *abort_flag != 0)) break;
-            }
-          }
-          if (!got) {
-            *abort_flag = 1;
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_slot_empty + 8 * slot, (use & 1) ^ 1, abort_flag))) {
             timed_out = true;
             break;
           }
           if (j < n_pre) {
-            {
-              // one lane per 64-column chunk: the copies are issued side by side
-              const CUtensorMap *map = kv ? &prm.vpre : &prm.kpre;
-              if (lane < G_::kChunks) tma_load_4d(dst + lane * kChunkBytes, map, full, lane * 64, j * kBlockN, it.hk, it.b);
-              if (lane == 0) mbar_arrive_expect_tx(full, G_::kTileBytes);
-            }
+            // one lane per 64-column chunk: the copies are issued side by side
+            const CUtensorMap *map = kv ? &prm.vpre : &prm.kpre;
+            if (lane < G_::kChunks) tma_load_4d(dst + lane * kChunkBytes, map, full, lane * 64, j * kBlockN, it.hk, it.b);
+            if (lane == 0) mbar_arrive_expect_tx(full, G_::kTileBytes);
           } else {
+            if (!list_seen && prm.idx_bstride == 0) {
+              int32_t *cache = reinterpret_cast<int32_t *>(smem + G_::kOffIdxCache);
+              list_ok = cache_shared_index_list(prm, cache, bad_index);
+              __syncwarp();
+              if (list_ok) idx_cache = cache;  // a malformed list is read entry by entry from global memory
+            }
+            list_seen = true;
             const int t0 = (j - n_pre) * kBlockN;
             const int n = min(kBlockN, prm.Lq - t0);
             if (kv == 1 && n < kBlockN) {
@@ -324,29 +298,59 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
             }
             // the V fill of a tile directly follows its K fill: the staged row list is still valid
             const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, kv ? &prm.v128 : &prm.k128, dst, kChunkBytes,
-                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, list_ok, bad_index, kv == 1);
+                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, list_ok, bad_index, kv == 1, true);
             if (lane == 0) mbar_arrive_expect_tx(full, bytes);
           }
           ++issued;
         }
       }
     }
-    // query tiles whose KV fills all went out before their buffer was released
-    while (!timed_out && q_next < n_my) {
-      bool ok = (q_next == 0) || mbar_wait(bar_q_free, (q_next - 1) & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) {
-        timed_out = true;
-        break;
-      }
-      issue_q(q_next);
-      ++q_next;
-    }
     if (timed_out) {
       // let copies already in flight land before the CTA's shared memory goes away
       for (int f = max(0, issued - G_::kSlots); f < issued; ++f)
         for (uint32_t w = 0; w < 4096 && !mbar_try_wait(bar_slot_full + 8 * (f % G_::kSlots), (f / G_::kSlots) & 1); ++w)
           __nanosleep(256);
+    }
+    if (bad_index && prm.status) atomicOr(prm.status, DS_DEV_INDEX);
+  } else if (warp == kQWarp) {
+    // ============================ TMA producer: query tiles ============================
+    // Item k's queries go to buffer q_buf(k) once the item that used it before (k - kQBufs) has issued its
+    // last Q K^T.  The row numbers are read from global memory here (every query tile is gathered once; the
+    // K/V producer's shared copy of the list may not exist yet).
+    bool bad_index = false;
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&prm.q32)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&prm.q1)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&prm.q128)) : "memory");
+    }
+    const int n_my = (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // items of this CTA
+    int k_done = 0;
+    for (int k = 0; k < n_my && !timed_out; ++k) {
+      if (k >= G_::kQBufs) {
+        if (!__all_sync(0xffffffffu, mbar_wait(q_free_bar(k), q_phase(k - G_::kQBufs), abort_flag))) {
+          timed_out = true;
+          break;
+        }
+      }
+      const Item it = decode_item<kSplit>(prm, blockIdx.x + k * gridDim.x);
+      const uint32_t full = q_full_bar(k);
+      uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ + q_buf(k) * G_::kTileBytes, kChunkBytes, full,
+                                      it.mt * kBlockM, it.m_rows, it.hk * prm.G, it.b, idxq_s, nullptr, false, bad_index, false, true);
+      if (it.x_rows > 0) {
+        // rows of the small query tile that are not loaded must be finite: clear the tile first
+        uint8_t *qx = smem + G_::kOffQx + q_buf(k) * G_::kQxBytes;
+        for (int q = lane; q < G_::kQxBytes / 16; q += 32) *reinterpret_cast<uint4 *>(qx + q * 16) = make_uint4(0, 0, 0, 0);
+        fence_proxy_async();
+        bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQx + q_buf(k) * G_::kQxBytes, kXChunkBytes, full,
+                                (it.mt + 1) * kBlockM, it.x_rows, it.hk * prm.G, it.b, idxq_s, nullptr, false, bad_index);
+      }
+      if (lane == 0) mbar_arrive_expect_tx(full, bytes);
+      k_done = k + 1;
+    }
+    if (timed_out) {
+      // let copies already in flight land before the CTA's shared memory goes away
+      for (int f = max(0, k_done - G_::kQBufs); f < k_done; ++f)
+        for (uint32_t w = 0; w < 4096 && !mbar_try_wait(q_full_bar(f), q_phase(f)); ++w) __nanosleep(256);
     }
     if (bad_index && prm.status) atomicOr(prm.status, DS_DEV_INDEX);
   } else if (warp == kMmaWarp) {
@@ -357,8 +361,8 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     constexpr uint32_t idesc_qk_x = instr_desc(kBlockM, kXRows, false, false);  // S_x^T = K Q_x^T
     const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
     // descriptors of byte 0 of each operand region; a K-step only adds to the address field
-    const uint64_t dq = smem_desc(sbase + G_::kOffQ, 16, 1024);
-    const uint64_t dqx = smem_desc(sbase + G_::kOffQx, 16, 1024);
+    const uint64_t dq0 = smem_desc(sbase + G_::kOffQ, 16, 1024);
+    const uint64_t dqx0 = smem_desc(sbase + G_::kOffQx, 16, 1024);
     const uint64_t dk0 = smem_desc(sbase + G_::kOffRing, 16, 1024);  // K tile, K-major
     bool ok = true;
     int g0 = 0;   // tiles processed by this CTA before the current item
@@ -369,7 +373,9 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       const int j_lo = kSplit ? decode_item<kSplit>(prm, item).t0 : 0;
       nt_cur = kSplit ? decode_item<kSplit>(prm, item).nt : n_tiles;
       const bool has_x = (D == 128) && decode_item<kSplit>(prm, item).x_rows > 0;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full, k & 1, abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(q_full_bar(k), q_phase(k), abort_flag));
+      const uint64_t dq = dq0 + (uint64_t)((q_buf(k) * G_::kTileBytes) >> 4);
+      const uint64_t dqx = dqx0 + (uint64_t)((q_buf(k) * G_::kQxBytes) >> 4);
       for (int jj = 0; jj < nt_cur && ok; ++jj) {
         const int j = j_lo + jj;
         (void)j;
@@ -419,7 +425,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
             umma_commit(bar_sx_full + 8 * (gx & 1));
           }
           umma_commit(bar_slot_empty + 8 * slot);
-          if (jj == nt_cur - 1) umma_commit(bar_q_free);
+          if (jj == nt_cur - 1) umma_commit(q_free_bar(k));
         }
         __syncwarp();
       }
@@ -934,6 +940,9 @@ int prepare_d(const ds_attn_params &p, AttnPrepared &out) {
   if (n_items > 0x7fffffffLL) return DS_ERR_UNSUPPORTED;
   prm.n_items = (int)n_items;
   out.grid = (int)(n_items < sm_count() ? n_items : sm_count());
+  // Two query buffers (and one ring slot fewer) pay when a CTA runs several items and the stall at an item
+  // boundary -- about two KV tiles' time with one buffer -- is a visible share of an item.
+  prm.q2 = (n_items > out.grid && n_tiles <= kQ2MaxTiles) ? 1 : 0;
   return DS_OK;
 }
 
@@ -943,11 +952,15 @@ int launch_prepared_d(const AttnPrepared &a, cudaStream_t stream) {
   // the attribute is per device: set it at every launch (cheap)
   const TcParams &prm = *reinterpret_cast<const TcParams *>(a.kernel_params);
   if (prm.splits > 1) {
-    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes));
-    attn_tc_kernel<D, true><<<a.grid, kNumThreads, Geo<D>::kSmemBytes, stream>>>(prm);
+    // every CTA has one item (a part of one): a second query buffer would have nothing to prefetch
+    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D, false>::kSmemBytes));
+    attn_tc_kernel<D, true, false><<<a.grid, kNumThreads, Geo<D, false>::kSmemBytes, stream>>>(prm);
+  } else if (prm.q2) {
+    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D, true>::kSmemBytes));
+    attn_tc_kernel<D, false, true><<<a.grid, kNumThreads, Geo<D, true>::kSmemBytes, stream>>>(prm);
   } else {
-    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes));
-    attn_tc_kernel<D, false><<<a.grid, kNumThreads, Geo<D>::kSmemBytes, stream>>>(prm);
+    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D, false>::kSmemBytes));
+    attn_tc_kernel<D, false, false><<<a.grid, kNumThreads, Geo<D, false>::kSmemBytes, stream>>>(prm);
   }
   DS_CUDA_OK(cudaGetLastError());
   note_launch(1);

@@ -169,10 +169,10 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
     auto issue_q = [&](int kq) {
       const Item2 it = decode_item2(prm, blockIdx.x + kq * gridDim.x);
       uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ, kChunkBytes, bar_q_full,
-                                      it.pr * 2 * kBlockM, it.rows_a, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index);
+                                      it.pr * 2 * kBlockM, it.rows_a, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index, false, true);
       if (it.rows_b > 0)
         bytes += gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ + G_::kTileBytes, kChunkBytes, bar_q_full,
-                                (it.pr * 2 + 1) * kBlockM, it.rows_b, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index);
+                                (it.pr * 2 + 1) * kBlockM, it.rows_b, it.hk * prm.G, it.b, idxq_s, idx_cache, list_ok, bad_index, false, true);
       if (lane == 0) mbar_arrive_expect_tx(bar_q_full, bytes);
     };
     int issued = 0;
@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(kThreads2, 1) attn_tc2_kernel(const __grid_con
               fence_proxy_async();
             }
             const uint32_t bytes = gather_rows<D>(prm, kv ? &prm.v32 : &prm.k32, kv ? &prm.v1 : &prm.k1, kv ? &prm.v128 : &prm.k128, dst, kChunkBytes,
-                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, list_ok, bad_index, kv == 1);
+                                                  full, t0, n, it.hk, it.b, idx_s, idx_cache, list_ok, bad_index, kv == 1, true);
             if (lane == 0) mbar_arrive_expect_tx(full, bytes);
           }
           ++issued;

@@ -82,6 +82,7 @@ __device__ __forceinline__ bool cache_shared_index_list(const AttnCommon &prm, i
 // Producer helper: fetch n gathered rows (logical rows R0 .. R0+n-1 of a stacked sequence whose
 // period is Lq) into a swizzled tile whose 64-column chunks are chunk_stride bytes apart.  The whole
 // warp calls it; lane 0 issues the copies (a whole-tile fetch: one lane per chunk).  Returns the bytes issued.
+// tile_end: the n rows are the last ones of their tile (whatever the copy writes behind them is not used).
 //
 // Runs of consecutive rows are fetched as one box (128 or 32 rows).  With list_ok (the list is known to be
 // strictly ascending and in range) the first and last entry of a run decide; otherwise every entry of the
@@ -91,7 +92,7 @@ template <int D>
 __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUtensorMap *map32, const CUtensorMap *map1,
                                                 const CUtensorMap *map128, uint32_t dst, uint32_t chunk_stride, uint32_t bar, int R0, int n,
                                                 int head0, int b, int32_t *idx_s, const int32_t *idx_cache, bool list_ok,
-                                                bool &bad_index, bool staged = false) {
+                                                bool &bad_index, bool staged = false, bool tile_end = false) {
   const int lane = threadIdx.x & 31;
   const int Lq = prm.Lq;
   const int32_t *ix = prm.idx + (long long)b * prm.idx_bstride;
@@ -104,21 +105,26 @@ __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUt
   // A full tile of consecutive rows inside one head (the current block and its window, every tile of a
   // cache-refresh step) needs no staging: one box per 64-column chunk fetches it, each chunk issued by a
   // lane of its own.
-  if (n == 128 && pos0 + 128 <= Lq) {
+  // The same box serves a shorter run when it is the last thing in the tile (so that the rows the box brings
+  // beyond the run overwrite nothing) and ends with the last row of the buffer: the box then reaches past the
+  // end of the tensor, where the copy fills in zeros.  That is every partial tile of compact buffers (T = Lq,
+  // idx = 0 .. Lq - 1), the layout ds_rope_gather produces.
+  // (Not for a handful of rows: the copy writes all 128 rows of the tile, zeros included.)
+  if (pos0 + n <= Lq && (n == 128 || (tile_end && n > 32))) {
     int first, last;
-    if (idx_cache != nullptr && pos0 + 127 < kIdxCap) {
+    if (idx_cache != nullptr && pos0 + n - 1 < kIdxCap) {
       first = idx_cache[pos0];
-      last = idx_cache[pos0 + 127];
+      last = idx_cache[pos0 + n - 1];
     } else {
       first = ix[pos0];
-      last = ix[pos0 + 127];
+      last = ix[pos0 + n - 1];
     }
-    bool whole = (last - first == 127 && first >= 0 && last < prm.T);
+    bool whole = (last - first == n - 1 && first >= 0 && last < prm.T) && (n == 128 || last == prm.T - 1);
     if (whole && !list_ok) {
-      // the order of the list is not known: all 128 entries must be the consecutive rows
+      // the order of the list is not known: all n entries must be the consecutive rows
       bool run = true;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) run = run && (ix[pos0 + lane + 32 * k] == first + lane + 32 * k);
+      for (int k = 0; k < 4; ++k) run = run && (lane + 32 * k >= n || ix[pos0 + lane + 32 * k] == first + lane + 32 * k);
       whole = __all_sync(0xffffffffu, run);
     }
     if (whole) {
@@ -159,6 +165,7 @@ __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUt
   }
   uint32_t bytes = 0;
   if (lane == 0) {
+    // one lane issues: the copies of an SM are taken one after the other whichever lanes issue them
     int r = 0, pos = pos0;
     while (r < n) {
       const int row = idx_s[r];
