@@ -192,6 +192,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
   const int n_tail = (prm.Lq + kBlockN - 1) / kBlockN;
   const int n_tiles = n_pre + n_tail;
 
+  const bool x_epilogue = prm.x_rows == 0;
   if (tid == 0) {
     mbar_init(bar_q_full, 1);
     mbar_init(bar_q_free, 1);
@@ -203,8 +204,10 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     mbar_init(bar_p_full + 8, kSoftmaxWarps);
     mbar_init(bar_pv_done, 1);
     mbar_init(bar_pv_done + 8, 1);
-    mbar_init(bar_o_free, kSoftmaxWarps);
-    mbar_init(bar_x, kXWarps);
+    // launches without extra rows: warps 10-13 write the items' results (see their role), so they are the ones
+    // that release O, and bar_x is the softmax warps' "row sums handed over"
+    mbar_init(bar_o_free, x_epilogue ? kXWarps : kSoftmaxWarps);
+    mbar_init(bar_x, x_epilogue ? kSoftmaxWarps : kXWarps);
     mbar_init(bar_x + 8, kXWarps);
     mbar_init(bar_y, kXWarps);
     mbar_init(bar_o_full, 1);
@@ -502,6 +505,58 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       }
     }
     timed_out = !ok;
+  } else if (warp >= kXWarp0 && warp < kXWarp0 + kXWarps && x_epilogue) {
+    // ============================ epilogue of the items (launches without extra rows) ============================
+    // The softmax warps leave each row's sum and maximum in shared memory and go straight on to the next item,
+    // whose first S tile is already waiting; these four warps, idle otherwise, wait for the item's last P V, read
+    // O (thread = row = TMEM lane), release it for the next item, normalise and store.  Measured before: from
+    // "last P stored" to the next item's first S tile the softmax warps spent about 5400 cycles against 300
+    // between two tiles of one item.
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const float *xl = reinterpret_cast<const float *>(smem + G_::kOffPx);  // [2 item parities][2: sum, maximum][128 rows]
+    bool ok = true;
+    int k = 0;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k) {
+      const Item it = decode_item<kSplit>(prm, item);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_x, k & 1, abort_flag));
+      if (!ok) break;
+      const float l_row = xl[((k & 1) * 2 + 0) * 128 + row], m_row = xl[((k & 1) * 2 + 1) * 128 + row];
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full, k & 1, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const bool live = row < it.m_rows;
+      const int R = it.mt * kBlockM + row;
+      const int hq = it.hk * prm.G + R / prm.Lq, i = R % prm.Lq;
+      const float inv = 1.f / l_row;
+      __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(prm.out) + (kSplit ? it.split * prm.out_split_stride : 0) + it.b * prm.out_stride[0] +
+                            hq * prm.out_stride[1] + (long long)i * prm.out_stride[2];
+#pragma unroll
+      for (int cb = 0; cb < D; cb += 32) {
+        uint32_t o[32];
+        tmem_ld32(lane_base + G_::kTmemO + cb, o);
+        tmem_wait_ld();
+        if (cb + 32 == D) {  // O is in registers: the next item's first P V may overwrite it
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_o_free);
+        }
+        if (live) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+            *reinterpret_cast<uint4 *>(orow + cb + c) = w;
+          }
+        }
+      }
+      if (live && prm.lse)
+        prm.lse[(kSplit ? it.split * prm.lse_split_stride : 0) + ((long long)it.b * prm.Hq + hq) * prm.Lq + i] = (m_row + log2f(l_row)) * kLn2;
+    }
+    timed_out = !ok;
   } else if (warp >= kXWarp0 && warp < kXWarp0 + kXWarps) {
     // ============================ transposed problem: softmax + epilogue ============================
     // Thread = key `row` of the tile (TMEM lane of S_x^T) and, for O_x^T, head-dimension element `row`.
@@ -775,6 +830,17 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       if (!ok) break;
       // ---- epilogue of the item ----
       l_sum += __shfl_xor_sync(0xffffffffu, l_sum, 16);
+      if (x_epilogue) {
+        // hand the row's sum and maximum to warps 10-13, which write the item's result, and go on
+        float *xl = reinterpret_cast<float *>(smem + G_::kOffPx);
+        if (half == 0) {
+          xl[((k & 1) * 2 + 0) * 128 + row] = l_sum;
+          xl[((k & 1) * 2 + 1) * 128 + row] = m_used;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_x);
+        continue;
+      }
       // the last P V of the item has completed (its own barrier, waited on once per item by everyone)
       ok = mbar_wait(bar_o_full, k & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);

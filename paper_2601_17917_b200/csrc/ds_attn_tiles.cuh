@@ -169,7 +169,7 @@ __device__ __forceinline__ uint32_t gather_rows(const AttnCommon &prm, const CUt
     int r = 0, pos = pos0;
     while (r < n) {
       const int row = idx_s[r];
-      const bool box32 = boxes && ((r & 7) == 0) && (r + 32 <= n) && (pos + 32 <= Lq) && (idx_s[r + 31] - row == 31);
+      const bool box32 = boxes && (r + 32 <= n) && (pos + 32 <= Lq) && (idx_s[r + 31] - row == 31);
       const int step = box32 ? 32 : 1;
 #pragma unroll
       for (int c = 0; c < (D / 64); ++c)

@@ -496,3 +496,44 @@ def test_few_work_items_split_over_the_keys(P, Lq, D):
     torch.cuda.synchronize()
     _compare(out3[1], ref[1], torch.bfloat16)
     assert (out3[0] == 9.0).all()
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,P,Lq,D", [
+    (25, 8, 8, 1100, 129, 128),     # 200 items of 11 KV tiles, one M-tile + one extra row each
+    (10, 60, 20, 1000, 43, 128),    # G = 3: 129 stacked rows, 200 items, extra row from another head
+    (5, 64, 32, 700, 150, 128),     # G = 2: 300 stacked rows = 3 M-tiles per KV head, no extra rows
+    (25, 8, 8, 1500, 64, 64),       # D = 64
+    (40, 4, 4, 2000, 136, 128),     # 8 extra rows
+])
+def test_more_items_than_sms_in_uneven_rounds(B, Hq, Hkv, P, Lq, D):
+    """More work items than SMs, in a number of rounds that leaves the last one mostly empty; items with and
+    without extra rows, stacked heads whose boundaries fall inside a tile, several M-tiles per KV head, D = 64.
+    Compared with the oracle on every element and with the log-sum-exp; then the same call restricted to listed
+    sequences with the count on the device (fewer items than the launch was sized for)."""
+    one = dict(kernel=ds.DS_ATTN_KERNEL_ONE_TILE)
+    T = Lq + 40
+    g = torch.Generator().manual_seed(B * 1000 + Lq)
+    mk = lambda *sh: torch.randn(*sh, generator=g).to(torch.bfloat16).to(DEV)
+    q, kt, vt, kp, vp = mk(B, Hq, T, D), mk(B, Hkv, T, D), mk(B, Hkv, T, D), mk(B, Hkv, P, D), mk(B, Hkv, P, D)
+    idx = np.arange(Lq, dtype=np.int32)
+    idx[-1] = T - 1
+    idx_t = torch.tensor(idx, device=DEV)
+    scale = 1.0 / math.sqrt(D)
+    out = torch.empty((B, Hq, Lq, D), dtype=torch.bfloat16, device=DEV)
+    ref, ref_lse = oracle.attn(_np(q), _np(kt), _np(vt), _np(kp), _np(vp), idx, scale, want_lse=True)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    lse = torch.empty((B, Hq, Lq), dtype=torch.float32, device=DEV)
+    ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, out=out, lse=lse, status=status, **one)
+    torch.cuda.synchronize()
+    assert ds.ds_read_status(status) == 0
+    _compare(out, ref, torch.bfloat16, f"rounds B{B} Hq{Hq} Hkv{Hkv} P{P} Lq{Lq} D{D}")
+    assert np.abs(lse.cpu().numpy() - ref_lse).max() < 2e-2
+    lst = torch.arange(B, dtype=torch.int32, device=DEV)
+    n_live = max(1, B // 3)
+    out2 = torch.full_like(out, 7.0)
+    ds.ds_attn_pruned(q, kt, vt, kp, vp, idx_t, scale, out=out2, status=status, seq_list=lst,
+                      n_seq_dev=torch.tensor([n_live], dtype=torch.int32, device=DEV), **one)
+    torch.cuda.synchronize()
+    assert ds.ds_read_status(status) == 0
+    _compare(out2[:n_live], ref[:n_live], torch.bfloat16, "rounds, listed sequences")
+    assert (out2[n_live:] == 7.0).all()
