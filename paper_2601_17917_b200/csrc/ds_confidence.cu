@@ -297,6 +297,8 @@ int launch_confidence_static(const void *logits, int dtype, int64_t rows, int64_
   if (n == 0) return DS_OK;
   if (n > kStaticRows) return DS_ERR_STATIC_LIMIT;
   const int splits = pick_splits(n, V, dtype);
+  // pick_splits keeps n * splits below 4 * SMs + n, far under the 2 * MAX_ROWS partial results the array holds
+  // for any n it accepts; the check only guards that arithmetic
   if (n * splits > kStaticPartials) return DS_ERR_STATIC_LIMIT;
   void *base = nullptr;
   const int rc = static_scratch(&base);
