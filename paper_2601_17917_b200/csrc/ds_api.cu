@@ -83,8 +83,8 @@ namespace ds {
 namespace {
 // Several M-tiles per KV head (wide windows, the unpruned reference, a cache-refresh step): the two-tile
 // kernel fetches every KV tile once for a pair of M-tiles and keeps the softmax warps busy on one tile while
-// the tensor pipe works for the other.  Measured per work item it costs about 1.85 single tiles for a full pair
-// and 1.05 for a pair with one tile (which alternates between the two S buffers like the one-tile kernel), so it
+// the tensor pipe works for the other.  Measured per work item it costs about 1.88 single tiles for a full pair
+// and 1.10 for a pair with one tile (which alternates between the two S buffers like the one-tile kernel), so it
 // pays when the number of rounds over the SMs does not grow.
 bool two_tile_kernel_pays(const ds_attn_params &p) {
   const long long rows = (long long)(p.Hq / p.Hkv) * p.Lq;
@@ -96,7 +96,7 @@ bool two_tile_kernel_pays(const ds_attn_params &p) {
   const long long heads = (long long)(p.seq_list ? p.n_seq : p.B) * p.Hkv, sms = sm_count();
   const double rounds1 = (double)((heads * n_mt1 + sms - 1) / sms);
   const double rounds2 = (double)((heads * n_pr + sms - 1) / sms);
-  const double pair_cost = (1.85 * (double)(n_mt / 2) + 1.05 * (double)(n_mt % 2)) / (double)n_pr;
+  const double pair_cost = (1.88 * (double)(n_mt / 2) + 1.10 * (double)(n_mt % 2)) / (double)n_pr;
   return rounds2 * pair_cost < 0.97 * rounds1;
 }
 
