@@ -4,7 +4,8 @@
 // Work item = (batch, KV head, 128-row M-tile).  The query heads of one GQA group are stacked along
 // M (row R = head_in_group * Lq + i), so every KV tile is read once per group.  KV is streamed as
 // 128-row tiles: first the cached prefix (tiled TMA boxes, out-of-range rows zero-filled), then the
-// retained tail rows named by the index list, fetched as 32-row TMA boxes where the list is
+// retained tail rows named by the index list, fetched as one 128-row box when a whole tile (or a
+// partial tile that ends with the buffer's last row) is consecutive, as 32-row boxes where the list is
 // contiguous and as single-row boxes elsewhere.  CTAs are persistent: CTA c takes items c, c + grid,
 // ... and the KV ring keeps streaming across item boundaries.
 //
@@ -17,15 +18,16 @@
 // moved (with an exact rescale) when a score exceeds it by more than 2^24.
 //
 // Warp roles (512 threads, one CTA per SM):
-//   warps 0-7  softmax + epilogue.  Warp w works on the 16 TMEM lanes 32 (w % 4) + 16 (w / 4) ..;
+//   warps 0-7  softmax (and, in launches with extra rows, the items' epilogue).  Warp w works on the 16 TMEM lanes 32 (w % 4) + 16 (w / 4) ..;
 //              two threads share a row (lanes l and l + 16 of the warp take the two column halves of
 //              every S tile, tcgen05.ld shape 16x32bx2), so a row maximum is one shuffle away and
 //              every scheduler has two softmax warps.
 //   warp  8    TMA producer of the K/V tiles (lane 0 issues; the warp stages the index list of each gathered tile)
 //   warp  9    TMEM allocation; issues Q K^T (one elected lane)
-//   warps 10-13 softmax + epilogue of the transposed problem (thread = key of the tile; idle in items
-//              without extra rows), kept apart so that its cross-warp agreement never sits on the
-//              main rows' critical path
+//   warps 10-13 softmax + epilogue of the transposed problem (thread = key of the tile), kept apart so that
+//              its cross-warp agreement never sits on the main rows' critical path.  In launches without
+//              extra rows they write the items' results instead (thread = row of the M-tile), so that the
+//              softmax warps can go straight on to the next item.
 //   warp 14    issues P V.  Issuing blocks while the tensor pipe's queue is full, so the two streams
 //              have an issuer each; the one dependency the pipe no longer orders by itself (Q K^T of
 //              tile g + 2 overwrites the buffer P V of tile g reads) is an explicit barrier wait.
