@@ -155,8 +155,11 @@ __device__ __forceinline__ Item decode_item(const TcParams &prm, int item) {
 // ------------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------------
-template <int D, bool kSplit, bool kQ2>
+// kX: the launch has rows beyond the last full M-tile (prm.x_rows > 0).  The two cases differ in what warps 10-13
+// and the epilogue do, and each instantiation carries only its own code.
+template <int D, bool kSplit, bool kQ2, bool kX>
 __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_constant__ TcParams prm) {
+  static_assert(!kX || D == 128, "extra rows exist for D = 128 only");
   using G_ = Geo<D, kQ2>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -194,7 +197,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
   const int n_tail = (prm.Lq + kBlockN - 1) / kBlockN;
   const int n_tiles = n_pre + n_tail;
 
-  const bool x_epilogue = prm.x_rows == 0;
+  constexpr bool x_epilogue = !kX;
   if (tid == 0) {
     mbar_init(bar_q_full, 1);
     mbar_init(bar_q_free, 1);
@@ -341,7 +344,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       const uint32_t full = q_full_bar(k);
       uint32_t bytes = gather_rows<D>(prm, &prm.q32, &prm.q1, &prm.q128, sbase + G_::kOffQ + q_buf(k) * G_::kTileBytes, kChunkBytes, full,
                                       it.mt * kBlockM, it.m_rows, it.hk * prm.G, it.b, idxq_s, nullptr, false, bad_index, false, true);
-      if (it.x_rows > 0) {
+      if (kX && it.x_rows > 0) {
         // rows of the small query tile that are not loaded must be finite: clear the tile first
         uint8_t *qx = smem + G_::kOffQx + q_buf(k) * G_::kQxBytes;
         for (int q = lane; q < G_::kQxBytes / 16; q += 32) *reinterpret_cast<uint4 *>(qx + q * 16) = make_uint4(0, 0, 0, 0);
@@ -377,7 +380,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += nt_cur) {
       const int j_lo = kSplit ? decode_item<kSplit>(prm, item).t0 : 0;
       nt_cur = kSplit ? decode_item<kSplit>(prm, item).nt : n_tiles;
-      const bool has_x = (D == 128) && decode_item<kSplit>(prm, item).x_rows > 0;
+      const bool has_x = kX && decode_item<kSplit>(prm, item).x_rows > 0;
       ok = __all_sync(0xffffffffu, mbar_wait(q_full_bar(k), q_phase(k), abort_flag));
       const uint64_t dq = dq0 + (uint64_t)((q_buf(k) * G_::kTileBytes) >> 4);
       const uint64_t dqx = dqx0 + (uint64_t)((q_buf(k) * G_::kQxBytes) >> 4);
@@ -452,7 +455,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k, g0 += nt_cur) {
       const int j_lo = kSplit ? decode_item<kSplit>(prm, item).t0 : 0;
       nt_cur = kSplit ? decode_item<kSplit>(prm, item).nt : n_tiles;
-      const bool has_x = (D == 128) && decode_item<kSplit>(prm, item).x_rows > 0;
+      const bool has_x = kX && decode_item<kSplit>(prm, item).x_rows > 0;
       for (int jj = 0; jj < nt_cur && ok; ++jj) {
         const int j = j_lo + jj;
         (void)j;
@@ -507,7 +510,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       }
     }
     timed_out = !ok;
-  } else if (warp >= kXWarp0 && warp < kXWarp0 + kXWarps && x_epilogue) {
+  } else if (x_epilogue && warp >= kXWarp0 && warp < kXWarp0 + kXWarps) {
     // ============================ epilogue of the items (launches without extra rows) ============================
     // The softmax warps leave each row's sum and maximum in shared memory and go straight on to the next item,
     // whose first S tile is already waiting; these four warps, idle otherwise, wait for the item's last P V, read
@@ -559,7 +562,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
         prm.lse[(kSplit ? it.split * prm.lse_split_stride : 0) + ((long long)it.b * prm.Hq + hq) * prm.Lq + i] = (m_row + log2f(l_row)) * kLn2;
     }
     timed_out = !ok;
-  } else if (warp >= kXWarp0 && warp < kXWarp0 + kXWarps) {
+  } else if (kX && warp >= kXWarp0 && warp < kXWarp0 + kXWarps) {
     // ============================ transposed problem: softmax + epilogue ============================
     // Thread = key `row` of the tile (TMEM lane of S_x^T) and, for O_x^T, head-dimension element `row`.
     // The kXMax columns are the extra query rows.
@@ -585,7 +588,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       const int j_lo = kSplit ? decode_item<kSplit>(prm, item).t0 : 0;
       nt_cur = kSplit ? decode_item<kSplit>(prm, item).nt : n_tiles;
       const Item it = decode_item<kSplit>(prm, item);
-      if (!((D == 128) && it.x_rows > 0)) {
+      if (!(kX && it.x_rows > 0)) {
         // nothing to do, but stay in step with the per-item barrier (a parity wait cannot skip phases)
         ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full, k & 1, abort_flag));
         continue;
@@ -832,7 +835,7 @@ __global__ void __launch_bounds__(kNumThreads, 1) attn_tc_kernel(const __grid_co
       if (!ok) break;
       // ---- epilogue of the item ----
       l_sum += __shfl_xor_sync(0xffffffffu, l_sum, 16);
-      if (x_epilogue) {
+      if constexpr (x_epilogue) {
         // hand the row's sum and maximum to warps 10-13, which write the item's result, and go on
         float *xl = reinterpret_cast<float *>(smem + G_::kOffPx);
         if (half == 0) {
@@ -1014,22 +1017,31 @@ int prepare_d(const ds_attn_params &p, AttnPrepared &out) {
   return DS_OK;
 }
 
+template <int D, bool kSplit, bool kQ2, bool kX>
+int launch_instance(const AttnPrepared &a, const TcParams &prm, cudaStream_t stream) {
+  // the attribute is per device: set it at every launch (cheap)
+  DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, kSplit, kQ2, kX>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D, kQ2>::kSmemBytes));
+  attn_tc_kernel<D, kSplit, kQ2, kX><<<a.grid, kNumThreads, Geo<D, kQ2>::kSmemBytes, stream>>>(prm);
+  return DS_OK;
+}
+template <int D, bool kX>
+int launch_mode(const AttnPrepared &a, const TcParams &prm, cudaStream_t stream) {
+  // split launches: every CTA has one item (a part of one), a second query buffer would have nothing to prefetch
+  if (prm.splits > 1) return launch_instance<D, true, false, kX>(a, prm, stream);
+  if (prm.q2) return launch_instance<D, false, true, kX>(a, prm, stream);
+  return launch_instance<D, false, false, kX>(a, prm, stream);
+}
+
 template <int D>
 int launch_prepared_d(const AttnPrepared &a, cudaStream_t stream) {
   if (a.grid == 0) return DS_OK;
-  // the attribute is per device: set it at every launch (cheap)
   const TcParams &prm = *reinterpret_cast<const TcParams *>(a.kernel_params);
-  if (prm.splits > 1) {
-    // every CTA has one item (a part of one): a second query buffer would have nothing to prefetch
-    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D, false>::kSmemBytes));
-    attn_tc_kernel<D, true, false><<<a.grid, kNumThreads, Geo<D, false>::kSmemBytes, stream>>>(prm);
-  } else if (prm.q2) {
-    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D, true>::kSmemBytes));
-    attn_tc_kernel<D, false, true><<<a.grid, kNumThreads, Geo<D, true>::kSmemBytes, stream>>>(prm);
-  } else {
-    DS_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<D, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D, false>::kSmemBytes));
-    attn_tc_kernel<D, false, false><<<a.grid, kNumThreads, Geo<D, false>::kSmemBytes, stream>>>(prm);
-  }
+  int rc;
+  if constexpr (D == 128)
+    rc = prm.x_rows > 0 ? launch_mode<D, true>(a, prm, stream) : launch_mode<D, false>(a, prm, stream);
+  else
+    rc = launch_mode<D, false>(a, prm, stream);
+  if (rc != DS_OK) return rc;
   DS_CUDA_OK(cudaGetLastError());
   note_launch(1);
   if (prm.splits > 1) {
