@@ -39,7 +39,7 @@ DEFAULT_CONFIG = "long32-w64"
 NCU_TRAFFIC: dict = {
     # captured on the batch-4 instance of the workload (the committed ncu summaries) and scaled by the items one launch
     # processes (x8: traffic is proportional to the rows streamed); set back to None when a kernel changes
-    "long32-w64": {"attn_bytes_per_launch": 8 * (281.25e6 + 3.92e6), "confidence_bytes_per_launch": 8 * (64.78e6 + 0.32e6)},
+    "long32-w64": {"attn_bytes_per_launch": 8 * (281.25e6 + 4.71e6), "confidence_bytes_per_launch": 8 * (64.78e6 + 0.32e6)},
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
